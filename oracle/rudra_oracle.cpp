@@ -1,0 +1,366 @@
+// Rudra parameter-server oracle: TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+//
+// A plain, slow, single-threaded CPU statement of what the parameter server of
+// arXiv 1509.04210 computes: the n-softsync protocol (Section 3.1, Eq. 5), the
+// scalar timestamp / staleness / vector clock bookkeeping (Section 3.1, Eq. 2),
+// the staleness-modulated learning rate (Section 5.1, Eq. 6), the weight update
+// (Eq. 1c / 3 / 4 / 5) and pullWeights (Section 2, Section 3.2).  Floating
+// point is carried in double and stored as fp32 (the paper's precision,
+// Section 4.2).  Nothing is blocked, fused, vectorised or threaded.
+//
+// This file shares no code with the CUDA library and is never linked into it.
+// Only tests, the smoke check and the benchmark's CPU-baseline leg use it.
+//
+// Parity status of the parts the paper does not write out:
+//   * momentum / weight-decay form         : parity unpinned by the paper
+//     (the paper names "momentum 0.9" and a "weight regularization penalty"
+//     in Section 4.2 but prints no formula); pinned only by closed forms of
+//     the reading stated at OraclePS::step below.
+//   * sigma = 0 floor in the per-gradient and group-mean rate policies
+//     (alpha0/sigma is undefined at sigma = 0)  : parity unpinned by the paper.
+//   * AdaGrad form (Section 5.5 names the method, prints no formula)
+//                                           : parity unpinned by the paper.
+// Everything else is pinned by Eq. 2-6 and the staleness sets printed in
+// Section 5.1 (see tests/).
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <deque>
+#include <vector>
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// Counter-based generator: SplitMix64 (Steele, Lea, Flood 2014), from its
+// published definition.  Each use draws from its own stream.
+// ---------------------------------------------------------------------------
+struct SplitMix64 {
+  uint64_t s;
+  explicit SplitMix64(uint64_t seed) : s(seed) {}
+  uint64_t next() {
+    s += 0x9E3779B97F4A7C15ull;
+    uint64_t z = s;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+  }
+};
+
+// Stream state for (seed, purpose, id): purposes are 1 = push-order
+// permutations, 2 = a learner's compute times.
+uint64_t stream_state(uint64_t seed, uint64_t purpose, uint64_t id) {
+  return seed ^ (purpose << 48) ^ id;
+}
+
+enum EventKind : int32_t {
+  EV_PUSH = 1,       // learner's gradient arrives; pulled_ts = timestamp of the weights it used
+  EV_STEP = 2,       // weights advance; ts = the new timestamp
+  EV_PULL = 3,       // learner receives the weights; ts = their timestamp
+  EV_PULL_SKIP = 4,  // timestamp inquiry found the learner's copy current (Section 3.2)
+  EV_BROADCAST = 5,  // every learner receives the weights with timestamp ts
+};
+
+enum SchedMode : int32_t {
+  MODE_HARDSYNC = 0,
+  MODE_SOFTSYNC_ROUNDS = 1,
+  MODE_SOFTSYNC_TIMED = 2,
+};
+
+struct Event {
+  int32_t kind;
+  uint32_t learner;
+  uint64_t pulled_ts;
+  uint64_t ts;
+  uint64_t seq;   // PUSH: index of this learner's mini-batch (0-based); else 0
+  uint64_t tick;  // simulated time of the event (timed mode), else the global push count
+};
+
+// ---------------------------------------------------------------------------
+// Learner event model (Section 2 learner loop; Section 3.2: a learner pulls
+// before each mini-batch, inquiring the timestamp first; the server handles
+// messages strictly one at a time).
+// ---------------------------------------------------------------------------
+struct OracleSched {
+  uint32_t lambda, n, c;
+  int32_t mode;
+  bool downcast;          // weights broadcast to every learner after each update (Section 3.3)
+  double ln_sigma;
+  uint64_t ts = 0;        // server timestamp, starts at 0 (Section 3.1)
+  uint64_t pushes = 0;    // gradients handled so far
+  std::vector<uint64_t> local_ts;   // timestamp of the weights last delivered to each learner
+  std::vector<uint64_t> grad_ts;    // timestamp of the weights its current mini-batch started from
+  std::vector<uint64_t> nbatch;     // mini-batches each learner has pushed
+  std::deque<Event> out;
+  // rounds
+  SplitMix64 perm_rng;
+  // timed
+  std::vector<SplitMix64> time_rng;
+  std::vector<uint64_t> next_push;
+
+  OracleSched(uint32_t lambda_, uint32_t n_, int32_t mode_, uint64_t seed, double ln_sigma_, bool downcast_)
+      : lambda(lambda_), n(n_), c(lambda_ / n_), mode(mode_), downcast(downcast_), ln_sigma(ln_sigma_),
+        local_ts(lambda_, 0), grad_ts(lambda_, 0), nbatch(lambda_, 0), perm_rng(stream_state(seed, 1, 0)) {
+    if (mode == MODE_SOFTSYNC_TIMED) {
+      for (uint32_t l = 0; l < lambda; ++l) time_rng.emplace_back(stream_state(seed, 2, l));
+      next_push.resize(lambda);
+      for (uint32_t l = 0; l < lambda; ++l) next_push[l] = draw_ticks(l);  // all start at time 0
+    }
+  }
+
+  // One compute time: lognormal(0, ln_sigma) in units of 2^-20, Box-Muller cosine branch.
+  uint64_t draw_ticks(uint32_t l) {
+    uint64_t a = time_rng[l].next() >> 11;
+    uint64_t b = time_rng[l].next() >> 11;
+    double u1 = (double)(a + 1) * 0x1.0p-53;   // (0, 1]
+    double u2 = (double)b * 0x1.0p-53;         // [0, 1)
+    double z = std::sqrt(-2.0 * std::log(u1)) * std::cos(6.283185307179586476925286766559 * u2);
+    long long t = std::llround(std::exp(ln_sigma * z) * 1048576.0);
+    return t < 1 ? 1ull : (uint64_t)t;
+  }
+
+  void emit(int32_t kind, uint32_t l, uint64_t pulled, uint64_t ts_, uint64_t seq, uint64_t tick) {
+    out.push_back(Event{kind, l, pulled, ts_, seq, tick});
+  }
+
+  // The server handles learner l's push completely -- including the update it
+  // may trigger -- before that learner's pull.
+  void handle_push(uint32_t l, uint64_t tick) {
+    emit(EV_PUSH, l, grad_ts[l], ts, nbatch[l], tick);
+    nbatch[l] += 1;
+    pushes += 1;
+    bool stepped = false;
+    if (pushes % c == 0) {          // exactly c gradients per update (Eq. 5)
+      ts += 1;                      // one increment per weight update (Section 3.1)
+      stepped = true;
+      emit(EV_STEP, l, 0, ts, 0, tick);
+    }
+    if (mode == MODE_HARDSYNC) {
+      if (stepped) {                // new weights go to all learners (Section 3.1, hardsync)
+        emit(EV_BROADCAST, 0, 0, ts, 0, tick);
+        for (uint32_t k = 0; k < lambda; ++k) local_ts[k] = grad_ts[k] = ts;   // all wait at the barrier
+      }
+      return;
+    }
+    if (stepped && downcast) {
+      // Weights reach every learner's receive buffer in the background; a learner in the middle
+      // of a mini-batch keeps computing on the weights it started from (Section 3.3).
+      emit(EV_BROADCAST, 0, 0, ts, 0, tick);
+      for (uint32_t k = 0; k < lambda; ++k) local_ts[k] = ts;
+    }
+    if (local_ts[l] == ts) {
+      emit(EV_PULL_SKIP, l, 0, ts, 0, tick);
+    } else {
+      local_ts[l] = ts;
+      emit(EV_PULL, l, 0, ts, 0, tick);
+    }
+    grad_ts[l] = local_ts[l];       // the learner starts its next mini-batch from these weights
+  }
+
+  void refill() {
+    if (mode == MODE_SOFTSYNC_TIMED) {
+      uint32_t best = 0;            // earliest push; ties go to the smaller learner id
+      for (uint32_t l = 1; l < lambda; ++l)
+        if (next_push[l] < next_push[best]) best = l;
+      uint64_t t = next_push[best];
+      handle_push(best, t);
+      next_push[best] = t + draw_ticks(best);
+      return;
+    }
+    // One round: every learner pushes exactly once, in a fresh seeded order.
+    std::vector<uint32_t> perm(lambda);
+    for (uint32_t i = 0; i < lambda; ++i) perm[i] = i;
+    for (uint32_t i = lambda - 1; i >= 1; --i) {
+      uint32_t j = (uint32_t)(perm_rng.next() % (uint64_t)(i + 1));
+      std::swap(perm[i], perm[j]);
+    }
+    for (uint32_t i = 0; i < lambda; ++i) handle_push(perm[i], pushes + 1);
+  }
+
+  Event next() {
+    while (out.empty()) refill();
+    Event e = out.front();
+    out.pop_front();
+    return e;
+  }
+};
+
+// ---------------------------------------------------------------------------
+// Parameter server state and the update rule.
+// ---------------------------------------------------------------------------
+enum LrPolicy : int32_t { LR_PAPER_N = 0, LR_PER_GRADIENT = 1, LR_GROUP_MEAN = 2 };
+enum GradDtype : int32_t { GRAD_F32 = 0, GRAD_BF16 = 1 };
+enum Optimizer : int32_t { OPT_MOMENTUM_SGD = 0, OPT_ADAGRAD = 1 };
+
+struct Pending {
+  const void* grad;
+  uint64_t pulled_ts;
+};
+
+struct OraclePS {
+  uint64_t N;
+  uint32_t lambda, n, c;
+  float alpha0, momentum, wd;
+  int32_t policy = LR_PAPER_N;
+  int32_t dtype = GRAD_F32;
+  int32_t optimizer = OPT_MOMENTUM_SGD;
+  float adagrad_eps = 1e-8f;
+  std::vector<float> theta, vel;   // vel: velocity (momentum SGD) or squared-gradient sum (AdaGrad)
+  uint64_t ts = 0;
+  std::deque<Pending> fifo;
+  // record of the most recent update
+  std::vector<uint64_t> clock;     // vector clock <p_1..p_c> (Section 3.1)
+  std::vector<uint32_t> sigma;
+  std::vector<float> scale;
+  float abar = 0.f;
+  double avg_sigma = 0.0;
+
+  OraclePS(uint64_t N_, uint32_t lambda_, uint32_t n_, float a0, float m, float wd_)
+      : N(N_), lambda(lambda_), n(n_), c(lambda_ / n_), alpha0(a0), momentum(m), wd(wd_),
+        theta(N_, 0.f), vel(N_, 0.f) {}
+
+  double grad_at(const void* g, uint64_t k) const {
+    if (dtype == GRAD_F32) return (double)((const float*)g)[k];
+    uint32_t bits = (uint32_t)((const uint16_t*)g)[k] << 16;   // bf16 is the top half of an fp32
+    float f;
+    std::memcpy(&f, &bits, 4);
+    return (double)f;
+  }
+
+  int64_t push(const void* g, uint64_t pulled_ts) {
+    if (pulled_ts > ts) return -2;          // weights with that timestamp do not exist yet (Section 3.1)
+    fifo.push_back(Pending{g, pulled_ts});
+    return (int64_t)fifo.size();
+  }
+
+  int step() {
+    if (fifo.size() < c) return 0;
+    std::vector<Pending> grp(fifo.begin(), fifo.begin() + c);
+    // staleness of each gradient: server timestamp j minus gradient timestamp i (Section 3.1)
+    clock.assign(c, 0);
+    sigma.assign(c, 0);
+    uint64_t sum_sigma = 0, sum_p = 0;
+    for (uint32_t l = 0; l < c; ++l) {
+      clock[l] = grp[l].pulled_ts;
+      sigma[l] = (uint32_t)(ts - grp[l].pulled_ts);
+      sum_sigma += sigma[l];
+      sum_p += grp[l].pulled_ts;
+    }
+    // Eq. 2: <sigma> = (i-1) - mean(i_1..i_c), (i-1) being the timestamp before this update.
+    avg_sigma = (double)ts - (double)sum_p / (double)c;
+    // Per-gradient step sizes: learning rate (Eq. 6, or a variant of it) times the 1/c of Eq. 5.
+    scale.assign(c, 0.f);
+    double sum_s = 0.0;
+    for (uint32_t l = 0; l < c; ++l) {
+      double div;
+      if (policy == LR_PAPER_N) {
+        div = (double)n * (double)c;                                   // alpha0 / n, Eq. 6
+      } else if (policy == LR_PER_GRADIENT) {
+        div = (double)std::max<uint32_t>(sigma[l], 1u) * (double)c;    // alpha0 / sigma_l (Section 5.1 footnote)
+      } else {
+        div = (double)std::max<uint64_t>(sum_sigma, (uint64_t)c);      // alpha0 / <sigma> of Eq. 2, then / c
+      }
+      scale[l] = (float)((double)alpha0 / div);
+      sum_s += (double)scale[l];
+    }
+    abar = (float)sum_s;   // the group's learning rate: sum of the per-gradient step sizes
+
+    for (uint64_t k = 0; k < N; ++k) {
+      if (optimizer == OPT_MOMENTUM_SGD) {
+        // sumGradients: staleness-scaled average of the c gradients (Eq. 5 with Eq. 6 folded in)
+        double acc = 0.0;
+        for (uint32_t l = 0; l < c; ++l) acc += (double)scale[l] * grad_at(grp[l].grad, k);
+        // applyUpdate, reading: L2 penalty joins the gradient at the group's rate; heavy-ball
+        // velocity carries the learning rate; with momentum = wd = 0 this is Eq. 5 exactly.
+        double u = acc + (double)abar * (double)wd * (double)theta[k];
+        double v = (double)momentum * (double)vel[k] + u;
+        double th = (double)theta[k] - v;
+        vel[k] = (float)v;
+        theta[k] = (float)th;
+      } else {
+        // AdaGrad at the server (Section 5.5), reading: the averaged gradient of Eq. 5 plus the
+        // L2 penalty feeds a running sum of squares; the step is rate * g / (sqrt(sum) + eps).
+        double gbar = 0.0;
+        for (uint32_t l = 0; l < c; ++l)
+          gbar += ((double)scale[l] / (double)abar) * grad_at(grp[l].grad, k);
+        gbar += (double)wd * (double)theta[k];
+        double h = (double)vel[k] + gbar * gbar;
+        double th = (double)theta[k] - (double)abar * gbar / (std::sqrt(h) + (double)adagrad_eps);
+        vel[k] = (float)h;
+        theta[k] = (float)th;
+      }
+    }
+    ts += 1;   // each weight update increments the timestamp by one (Section 3.1)
+    fifo.erase(fifo.begin(), fifo.begin() + c);
+    return 1;
+  }
+
+  int64_t pull(float* dst) const {   // pullWeights: the weights and their timestamp (Section 3.2)
+    for (uint64_t k = 0; k < N; ++k) dst[k] = theta[k];
+    return (int64_t)ts;
+  }
+};
+
+}  // namespace
+
+extern "C" {
+
+void ora_splitmix64(uint64_t seed, uint64_t count, uint64_t* out) {
+  SplitMix64 g(seed);
+  for (uint64_t i = 0; i < count; ++i) out[i] = g.next();
+}
+
+void* ora_sched_create(uint32_t lambda, uint32_t n, int32_t mode, uint64_t seed, double ln_sigma, int32_t downcast) {
+  if (lambda == 0 || n == 0 || n > lambda) return nullptr;
+  if (mode < 0 || mode > 2) return nullptr;
+  if (mode == MODE_HARDSYNC && n != 1) return nullptr;
+  return new OracleSched(lambda, n, mode, seed, ln_sigma, downcast != 0);
+}
+void ora_sched_destroy(void* s) { delete (OracleSched*)s; }
+// Writes count events into out (6 x 8-byte fields each: kind|learner packed as two 32-bit words,
+// pulled_ts, ts, seq, tick).
+void ora_sched_run(void* s, uint64_t count, Event* out) {
+  OracleSched* S = (OracleSched*)s;
+  for (uint64_t i = 0; i < count; ++i) out[i] = S->next();
+}
+
+void* ora_ps_create(uint64_t N, uint32_t lambda, uint32_t n, float alpha0, float momentum, float wd) {
+  if (N == 0 || lambda == 0 || n == 0 || n > lambda) return nullptr;
+  return new OraclePS(N, lambda, n, alpha0, momentum, wd);
+}
+void ora_ps_destroy(void* p) { delete (OraclePS*)p; }
+void ora_ps_set_policy(void* p, int32_t policy) { ((OraclePS*)p)->policy = policy; }
+void ora_ps_set_grad_dtype(void* p, int32_t dtype) { ((OraclePS*)p)->dtype = dtype; }
+void ora_ps_set_optimizer(void* p, int32_t opt, float eps) {
+  ((OraclePS*)p)->optimizer = opt;
+  ((OraclePS*)p)->adagrad_eps = eps;
+}
+void ora_ps_set_alpha0(void* p, float a0) { ((OraclePS*)p)->alpha0 = a0; }
+void ora_ps_set_weights(void* p, const float* src) {
+  OraclePS* P = (OraclePS*)p;
+  for (uint64_t k = 0; k < P->N; ++k) { P->theta[k] = src[k]; P->vel[k] = 0.f; }
+  P->ts = 0;
+  P->fifo.clear();
+}
+int64_t ora_ps_push(void* p, const void* grad, uint64_t pulled_ts) { return ((OraclePS*)p)->push(grad, pulled_ts); }
+int32_t ora_ps_step(void* p) { return ((OraclePS*)p)->step(); }
+int64_t ora_ps_pull(void* p, float* dst) { return ((OraclePS*)p)->pull(dst); }
+int64_t ora_ps_timestamp(void* p) { return (int64_t)((OraclePS*)p)->ts; }
+void ora_ps_state(void* p, float* vel_out) {
+  OraclePS* P = (OraclePS*)p;
+  for (uint64_t k = 0; k < P->N; ++k) vel_out[k] = P->vel[k];
+}
+int32_t ora_ps_last_clock(void* p, uint64_t* pulled, uint32_t* sigma, float* scale, double* avg_sigma, float* abar) {
+  OraclePS* P = (OraclePS*)p;
+  uint32_t c = (uint32_t)P->clock.size();
+  for (uint32_t l = 0; l < c; ++l) {
+    if (pulled) pulled[l] = P->clock[l];
+    if (sigma) sigma[l] = P->sigma[l];
+    if (scale) scale[l] = P->scale[l];
+  }
+  if (avg_sigma) *avg_sigma = P->avg_sigma;
+  if (abar) *abar = P->abar;
+  return (int32_t)c;
+}
+
+}  // extern "C"
