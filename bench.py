@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the parameter-server update path: updates/s and achieved HBM bandwidth.
+
+One step = one update window of the learner event stream: the c = floor(lambda/n) pushGradient
+messages of a group, the fused sumGradients + applyUpdate launch, and the pullWeights copies the
+learners of that window make.  Default workload: the ImageNet-scale model (60 965 224 fp32
+weights, lambda = 54, n = 18, c = 3, momentum 0.9, weight decay 5e-4) on synthetic gradient
+streams, one distinct buffer per learner so every byte comes from HBM.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+With N > 1 (under torchrun) every rank runs an independent replica of the server: the path has
+no exchange step on one node, so there is no collective in the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1509_04210_b200 import synth  # noqa: E402
+
+METRIC = "ps_updates_per_sec"
+UNIT = "updates/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def update_bytes_per_param(w):
+    """Algorithmic bytes one update moves per weight: c gradient reads + read and write of the
+    weights and (with momentum) of the velocity."""
+    g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
+    return w.c * g + (16 if w.momentum != 0.0 else 8)
+
+
+EV_PUSH, EV_STEP, EV_PULL, EV_PULL_SKIP, EV_BROADCAST = 1, 2, 3, 4, 5
+
+
+def make_windows(w, count, seed=synth.MASTER_SEED, from_oracle=False):
+    """Event windows: a window runs from the first push of a group to the last pull before the
+    next group's first push.  The CUDA arm takes the events from the library's scheduler, the
+    reference arm from the oracle's."""
+    if from_oracle:
+        from oracle import rudra_oracle as ora
+
+        osched = ora.OracleScheduler(w.lam, w.n, w.mode, seed, w.lognormal_sigma, w.downcast)
+        next_event = lambda: osched.run(1)[0]
+    else:
+        from paper_1509_04210_b200 import binding as rb
+
+        sched = rb.Scheduler(w.lam, w.n, w.mode, seed, w.lognormal_sigma, w.downcast)
+        next_event = lambda: sched.next(1)[0]
+    windows, cur, stepped = [], [], False
+    while len(windows) < count:
+        ev = next_event()
+        kind = int(ev["kind"])
+        if kind == EV_PUSH and stepped:
+            windows.append(cur)
+            cur, stepped = [], False
+        cur.append((kind, int(ev["learner"]), int(ev["pulled_ts"]), int(ev["ts"])))
+        if kind == EV_STEP:
+            stepped = True
+    return windows
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons while the timed region runs (read-only NVML queries)."""
+
+    def __init__(self, index, period=0.005):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reasons, self.max_mhz = period, [], set(), None
+        self._halt = threading.Event()
+        self._h = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def run(self):
+        if self._h is None:
+            return
+        nv = self._nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._halt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=2.0)
+        return {
+            "sm_mhz": float(np.median(self.samples)) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+def visible_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs (the reported baseline and the --impl reference arm)
+# ---------------------------------------------------------------------------------------------
+def oracle_run(w, windows, nsample, grads_host, warmup=0, budget_s=None, max_windows=None):
+    """Times the oracle, as it stands, over event windows (from the start of the event stream) on
+    the first nsample weights; the first ``warmup`` windows run untimed."""
+    from oracle import rudra_oracle as ora
+
+    ps = ora.OraclePS(nsample, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
+    ps.set_grad_dtype(w.grad_dtype)
+    ps.set_weights(synth.initial_weights(nsample, w.theta_std))
+    done, t0 = -warmup, time.perf_counter()
+    for win in windows:
+        if done == 0:
+            t0 = time.perf_counter()
+        for kind, learner, pulled_ts, ts in win:
+            if kind == ora.PUSH:
+                ps.push(grads_host[learner % len(grads_host)], pulled_ts)
+            elif kind == ora.STEP:
+                ps.step()
+            elif kind == ora.PULL:
+                ps.pull()
+            elif kind == ora.BROADCAST:
+                for _ in range(w.lam):
+                    ps.pull()
+        done += 1
+        if max_windows is not None and done >= max_windows:
+            break
+        if budget_s is not None and time.perf_counter() - t0 >= budget_s:
+            break
+    return done, time.perf_counter() - t0
+
+
+def host_gradients(w, nsample, count):
+    return [synth.gradient(nsample, l, 0, w.grad_std, w.grad_dtype) for l in range(count)]
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle on the same workload, metric and unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import rudra_oracle as ora
+
+    ora.build()
+    nsample = max(1, w.nparams // 4) if w.nparams > (1 << 22) else w.nparams
+    windows = make_windows(w, args.warmup + args.steps, from_oracle=True)
+    grads = host_gradients(w, nsample, min(w.lam, 8))
+    done, dt = oracle_run(w, windows, nsample, grads, warmup=args.warmup)
+    frac = nsample / w.nparams
+    value = done / dt * frac
+    sample = "first %d of %d weights (%.0f%%), %d distinct host gradient buffers, rate scaled by the fraction" % (
+        nsample, w.nparams, 100 * frac, len(grads))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w):
+    return {
+        "workload": w.name, "nparams": w.nparams, "lambda": w.lam, "n": w.n, "c": w.c, "alpha0": w.alpha0,
+        "momentum": w.momentum, "weight_decay": w.weight_decay,
+        "grad_dtype": "bf16" if w.grad_dtype == synth.GRAD_BF16 else "f32",
+        "scheduler": {0: "hardsync", 1: "softsync_rounds", 2: "softsync_timed"}[w.mode],
+        "l2": "inputs larger than L2: one distinct gradient buffer per learner, %.2f GB touched per update window"
+              % ((update_bytes_per_param(w) + 8 * w.c) * w.nparams / 1e9),
+        "parallelism": "replicas",
+    }
+
+
+# ---------------------------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_1509_04210_b200 import binding as rb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    rb.lib()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    N = w.nparams
+    seed = synth.MASTER_SEED + rank
+    stream = torch.cuda.Stream()
+    bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype, seed) for l in range(w.lam)]
+    nslots = w.lam
+    slots = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(nslots)]
+    ps = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
+    ps.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
+    ps.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
+    ps.sync()
+    ps.set_stream(stream)
+    windows = make_windows(w, args.warmup + args.steps)
+
+    def run_window(win, ev_pairs=None):
+        for kind, learner, pulled_ts, ts in win:
+            if kind == rb.EV_PUSH:
+                ps.push(bufs[learner], pulled_ts)
+            elif kind == rb.EV_STEP:
+                if ev_pairs is not None:
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    ps.step()
+                    e1.record(stream)
+                    ev_pairs.append((e0, e1))
+                else:
+                    ps.step()
+            elif kind == rb.EV_PULL:
+                ps.pull(slots[learner])
+            elif kind == rb.EV_BROADCAST:
+                ps.pull_many(slots)
+
+    for win in windows[: args.warmup]:
+        run_window(win)
+    barrier()
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()
+    c0 = ps.counters()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pairs = []
+    start.record(stream)
+    for win in windows[args.warmup:]:
+        run_window(win, pairs)
+    end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    c1 = ps.counters()
+    ms = start.elapsed_time(end)
+    upd_ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+    launches = c1["launches"] - c0["launches"]
+    pulls = c1["pulls"] - c0["pulls"]
+
+    # end to end through the C interface with host buffers: gradients travel host -> device inside
+    # the timed region and every pulled copy of the weights travels device -> host
+    e2e_steps = min(args.steps, 16 if N > (1 << 24) else 200)
+    nhost = min(w.lam, 8)
+    hg = []
+    for l in range(nhost):
+        t = torch.empty(N, dtype=bufs[0].dtype).pin_memory()
+        t.copy_(bufs[l])
+        hg.append(t)
+    hdst = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(2)]
+    torch.cuda.synchronize()
+    ps2 = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
+    ps2.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
+    ps2.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
+    ps2.sync()
+    ps2.set_stream(stream)
+
+    def run_window_host(win):
+        k = 0
+        for kind, learner, pulled_ts, ts in win:
+            if kind == rb.EV_PUSH:
+                ps2.push_host(hg[learner % nhost], pulled_ts)
+            elif kind == rb.EV_STEP:
+                ps2.step()
+            elif kind == rb.EV_PULL:
+                ps2.pull_host(hdst[k % 2])
+                k += 1
+            elif kind == rb.EV_BROADCAST:
+                ps2.pull_host(hdst[0])   # one copy leaves the device; learners on the host share it
+
+    e2e_warm = min(args.warmup, 3)
+    for win in windows[:e2e_warm]:
+        run_window_host(win)
+    barrier()
+    h0 = ps2.counters()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record(stream)
+    for win in windows[e2e_warm: e2e_warm + e2e_steps]:
+        run_window_host(win)
+    e2.record(stream)
+    barrier()
+    h1 = ps2.counters()
+    e2e_ms = s2.elapsed_time(e2)
+    ps2.close()
+
+    times = torch.tensor([ms, e2e_ms, upd_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms, e2e_ms, upd_ms = (float(x) for x in times.cpu())
+
+    if rank == 0:
+        peak, peak_kind = measured_hbm_peak()
+        bpp = update_bytes_per_param(w)
+        upd_bytes = bpp * N
+        achieved = upd_bytes / (upd_ms * 1e-3) / 1e9
+        window_bytes = (upd_bytes * args.steps + 8 * N * pulls) / args.steps
+        value = world * args.steps / (ms * 1e-3)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(w),
+            "hbm_gbs_whole_path": window_bytes / (ms / args.steps * 1e-3) / 1e9,
+            "pulls_per_step": pulls / args.steps,
+            "update_kernel_updates_per_sec": 1e3 / upd_ms,
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "e2e": {
+                "value": world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                "h2d_bytes_per_step": (h1["h2d_bytes"] - h0["h2d_bytes"]) // e2e_steps,
+                "d2h_bytes_per_step": (h1["d2h_bytes"] - h0["d2h_bytes"]) // e2e_steps,
+            },
+            "roofline": {
+                "kernel": "update_kernel (fused sumGradients + applyUpdate)", "bound": "hbm",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": "of %s" % peak_kind, "bytes_per_param": bpp, "avg_launch_us": upd_ms * 1e3,
+                "frac_of_8TBs_datasheet": achieved / 8000.0,
+                "traffic": None,
+            },
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            from oracle import rudra_oracle as ora
+
+            ora.build()
+            nh = min(w.lam, 6)
+            grads = [t.cpu().numpy() if w.grad_dtype == synth.GRAD_F32 else t.view(torch.int16).cpu().numpy().view(np.uint16)
+                     for t in bufs[:nh]]
+            done, dt = oracle_run(w, windows, N, grads, warmup=1, budget_s=12.0, max_windows=args.steps)
+            line["cpu_baseline"] = {
+                "value": done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "sample": "%d full-size update windows of the same event stream (%d distinct gradient buffers), %.1f s"
+                          % (done, nh, dt),
+                "host_cores_available": os.cpu_count(),
+            }
+        print(json.dumps(line), flush=True)
+    ps.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="imagenet", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

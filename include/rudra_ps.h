@@ -1,0 +1,202 @@
+/*
+ * rudra_ps.h -- C interface of the B200 parameter-server update path of the Rudra framework
+ * (Gupta, Zhang, Wang, "Model Accuracy and Runtime Tradeoff in Distributed Deep Learning: A
+ * Systematic Study", arXiv 1509.04210).
+ *
+ * The server of Section 2 does two things: sumGradients (receive and accumulate the learners'
+ * gradients) and applyUpdate (multiply the accumulated gradient by the learning rate and update
+ * the weights, Eq. 1c).  Under the n-softsync protocol of Section 3.1 (Eq. 5) it updates after
+ * collecting c = floor(lambda / n) gradients, averaging them; every update raises a scalar
+ * weight timestamp by one, a gradient carries the timestamp of the weights it was computed
+ * from, and its staleness sigma is the server's timestamp minus the gradient's (Section 3.1).
+ * The learning rate is divided by the staleness (Section 3.2; Eq. 6: alpha = alpha0 / n).
+ * pullWeights hands a learner the weights and their timestamp (Section 2, Section 3.2).
+ *
+ * Conventions
+ *   - Plain C, no exceptions cross this boundary, the library never aborts the process.
+ *   - "dev" pointers are CUDA device addresses on the device that was current at create time;
+ *     "host" pointers are ordinary (preferably page-locked) host addresses.
+ *   - Every device vector is flat and contiguous and must start on a 32-byte boundary (the
+ *     kernels move 256 bits per access).
+ *   - Return values: >= 0 success, < 0 one of the RUDRA_E_* codes; rudra_last_error() gives
+ *     the reason as text.
+ *   - All device work is enqueued on the handle's stream and is asynchronous to the host;
+ *     only rudra_ps_sync and rudra_ps_destroy wait for the device.  The kernels contain no
+ *     waits, flags or inter-block communication.
+ *   - A handle is not thread-safe (the server of Section 3.2 handles messages one at a time);
+ *     distinct handles are independent.
+ *   - There is no CPU implementation behind these calls.
+ */
+#ifndef RUDRA_PS_H
+#define RUDRA_PS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rudra_ps rudra_ps;
+typedef struct rudra_sched rudra_sched;
+
+/* error codes */
+#define RUDRA_E_INVAL      (-1) /* null / misaligned pointer, bad argument, bad handle          */
+#define RUDRA_E_BAD_TS     (-2) /* pulled_ts is ahead of the server timestamp                    */
+#define RUDRA_E_QUEUE_FULL (-3) /* more than RUDRA_QUEUE_CAP gradients waiting                   */
+#define RUDRA_E_CUDA       (-4) /* a CUDA call failed; text in rudra_last_error()                */
+#define RUDRA_E_STATE      (-5) /* call not legal in the current state (e.g. queue not empty)    */
+
+#define RUDRA_MAX_GROUP  128    /* largest c = floor(lambda / n) one update can combine          */
+#define RUDRA_MAX_DSTS   128    /* most destinations of one pull_many / step_pull_many           */
+#define RUDRA_QUEUE_CAP  4096   /* most gradients that may wait in the queue                     */
+
+/* rudra_ps_set_option keys and values */
+#define RUDRA_OPT_GRAD_DTYPE 1
+#define   RUDRA_GRAD_F32  0     /* gradients are float (the paper's precision, Section 4.2)      */
+#define   RUDRA_GRAD_BF16 1     /* gradients are bfloat16; weights and state stay float          */
+#define RUDRA_OPT_LR_POLICY 2
+#define   RUDRA_LR_PAPER_N      0 /* alpha = alpha0 / n for every gradient (Eq. 6)               */
+#define   RUDRA_LR_PER_GRADIENT 1 /* alpha_l = alpha0 / max(sigma_l, 1) (Section 5.1, footnote)  */
+#define   RUDRA_LR_GROUP_MEAN   2 /* alpha = alpha0 / max(<sigma>, 1), <sigma> of Eq. 2          */
+#define RUDRA_OPT_OPTIMIZER 3
+#define   RUDRA_OPTIM_MOMENTUM_SGD 0 /* momentum-accelerated SGD with weight decay (Section 4.2) */
+#define   RUDRA_OPTIM_ADAGRAD      1 /* AdaGrad at the server (Section 5.5)                      */
+
+/*
+ * rudra_ps_create -- a parameter server for a flat model of nparams weights, lambda learners and
+ * splitting parameter n (Section 3.1: 1 <= n <= lambda, c = floor(lambda / n) gradients per
+ * update).  alpha0 is the base learning rate of Eq. 6, momentum and weight_decay those of
+ * Section 4.2.  Allocates the weights and one state vector (fp32, zeroed) on the current device;
+ * timestamp = 0.  Returns NULL on invalid arguments (nparams == 0, lambda == 0, n == 0,
+ * n > lambda, c > RUDRA_MAX_GROUP, negative or non-finite alpha0 / momentum / weight_decay,
+ * momentum >= 1) or CUDA failure.
+ */
+rudra_ps* rudra_ps_create(uint64_t nparams, uint32_t lambda, uint32_t n,
+                          float alpha0, float momentum, float weight_decay);
+
+/* Frees everything the handle owns after waiting for its stream.  NULL is a no-op. */
+void rudra_ps_destroy(rudra_ps* ps);
+
+/* All later device work of this handle goes to cuda_stream (a cudaStream_t / CUstream value,
+ * e.g. torch.cuda.Stream().cuda_stream); NULL selects the legacy default stream. */
+int rudra_ps_set_stream(rudra_ps* ps, void* cuda_stream);
+
+/* Sets one RUDRA_OPT_* key.  Only legal while no gradient is queued (else RUDRA_E_STATE).
+ * Changing the optimizer zeroes the state vector. */
+int rudra_ps_set_option(rudra_ps* ps, int key, int64_t value);
+
+/* Base learning rate for later updates (the step schedule of Section 4.2 divides it by 10). */
+int rudra_ps_set_alpha0(rudra_ps* ps, float alpha0);
+
+/* Copies nparams floats from src into the weights, zeroes the state, resets the timestamp to 0
+ * and empties the queue.  src_dev: device memory; src_host: host memory (copied on the stream). */
+int rudra_ps_set_weights(rudra_ps* ps, const float* src_dev);
+int rudra_ps_set_weights_host(rudra_ps* ps, const float* src_host);
+
+/*
+ * rudra_ps_push -- pushGradient as the server sees it (Section 2; Section 3.2: the message is the
+ * gradient plus the timestamp of the weights it was computed from).  grad_dev: nparams elements
+ * of the configured gradient type in device memory.  The buffer is BORROWED: it is read by the
+ * update that consumes it and must stay valid and unchanged until that update has run on the
+ * stream (re-use ordered on the same stream is safe).  pulled_ts must not exceed the server's
+ * timestamp (RUDRA_E_BAD_TS).  Returns the number of gradients now queued.  No device work.
+ */
+int64_t rudra_ps_push(rudra_ps* ps, const void* grad_dev, uint64_t pulled_ts);
+
+/* Same, for a gradient in host memory: it is copied on the stream into a staging buffer the
+ * handle owns (allocated on first use, re-used afterwards), so grad_host may be re-used once the
+ * copy has run.  Page-locked memory makes the copy asynchronous. */
+int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_ts);
+
+/*
+ * rudra_ps_step -- one weight update if at least c gradients are queued (Eq. 5): takes the c
+ * oldest, fixes sigma_l = timestamp - pulled_ts_l (Section 3.1), records the vector clock and
+ * <sigma> (Eq. 2), forms the per-gradient step sizes s_l = alpha_l / c (Eq. 5, Eq. 6), enqueues
+ * ONE fused kernel that computes, per weight k,
+ *     acc = sum_l s_l * g_l[k];  u = acc + (sum_l s_l) * weight_decay * theta[k];
+ *     v[k] = momentum * v[k] + u;  theta[k] -= v[k]
+ * and raises the timestamp by one.  Returns 1 if an update was enqueued, 0 if fewer than c
+ * gradients wait (nothing changes), < 0 on error.
+ */
+int rudra_ps_step(rudra_ps* ps);
+
+/* Like rudra_ps_step, and the same kernel also writes the new weights into k learner buffers
+ * (dsts_dev: host array of k device pointers, each nparams floats, 0 <= k <= RUDRA_MAX_DSTS):
+ * the update followed by k pulls at the cost of one read of the weights.  Section 3.1's hardsync
+ * broadcast and Section 3.3's weight down-cast are this call with k = lambda. */
+int rudra_ps_step_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k);
+
+/*
+ * rudra_ps_pull -- pullWeights (Section 2, Section 3.2): enqueues a copy of the weights, as of
+ * every update issued so far, into dst (caller-owned, nparams floats) and returns their
+ * timestamp.  rudra_ps_pull_host copies to host memory.  rudra_ps_pull_many serves k learners
+ * with one read of the weights.
+ */
+int64_t rudra_ps_pull(rudra_ps* ps, float* dst_dev);
+int64_t rudra_ps_pull_host(rudra_ps* ps, float* dst_host);
+int64_t rudra_ps_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k);
+
+/* The timestamp inquiry of Section 3.2: a learner whose copy already has this timestamp skips
+ * the pull.  Host only. */
+int64_t rudra_ps_timestamp(const rudra_ps* ps);
+
+/* Vector clock of the most recent update (Section 3.1): the c gradient timestamps, their
+ * staleness, the step sizes s_l used, and <sigma> of Eq. 2.  Any output may be NULL.  Returns c,
+ * or 0 before the first update. */
+int rudra_ps_last_clock(const rudra_ps* ps, uint64_t* pulled_ts_out, uint32_t* sigma_out,
+                        float* scale_out, double* avg_sigma_out);
+
+/* Checkpoint hooks: device-to-device copies of the weights and the state vector (either may be
+ * NULL) out of / into the handle; import also sets the timestamp and empties the queue. */
+int rudra_ps_export_state(rudra_ps* ps, float* theta_dst_dev, float* state_dst_dev);
+int rudra_ps_import_state(rudra_ps* ps, const float* theta_src_dev, const float* state_src_dev, uint64_t ts);
+
+/* Waits for the handle's stream; reports asynchronous CUDA errors as RUDRA_E_CUDA. */
+int rudra_ps_sync(rudra_ps* ps);
+
+/* Counters since create: out[0] pushes, out[1] updates, out[2] pulls served (destinations),
+ * out[3] kernels launched, out[4] bytes copied host->device, out[5] bytes copied device->host. */
+int rudra_ps_counters(const rudra_ps* ps, uint64_t out[6]);
+
+/* Reason of the calling thread's most recent failure; static storage, never freed. */
+const char* rudra_last_error(void);
+
+/* ------------------------------------------------------------------------------------------
+ * Learner event model.  The paper's server handles incoming messages strictly one by one
+ * (Section 3.2), which makes the arrival order the whole control; this host-only scheduler
+ * produces that order for lambda simulated learners running the loop of Section 2
+ * (pull, compute, push), with the timestamp inquiry of Section 3.2.
+ * ------------------------------------------------------------------------------------------ */
+#define RUDRA_EV_PUSH      1 /* learner's gradient arrives; pulled_ts = timestamp it carries      */
+#define RUDRA_EV_STEP      2 /* the c-th gradient of a group arrived: update; ts = new timestamp  */
+#define RUDRA_EV_PULL      3 /* learner receives the weights with timestamp ts                    */
+#define RUDRA_EV_PULL_SKIP 4 /* inquiry found the learner's copy current: no copy                 */
+#define RUDRA_EV_BROADCAST 5 /* all lambda learners receive the weights with timestamp ts         */
+
+#define RUDRA_SCHED_HARDSYNC        0 /* Section 3.1 hardsync: n = 1, barrier, broadcast          */
+#define RUDRA_SCHED_SOFTSYNC_ROUNDS 1 /* every learner pushes once per round, seeded order        */
+#define RUDRA_SCHED_SOFTSYNC_TIMED  2 /* learners with seeded lognormal compute times             */
+
+typedef struct rudra_event {
+  int32_t  kind;       /* RUDRA_EV_*                                                            */
+  uint32_t learner;    /* learner the event belongs to (STEP: whose push closed the group)      */
+  uint64_t pulled_ts;  /* PUSH: timestamp of the weights the gradient was computed from         */
+  uint64_t ts;         /* PUSH: server timestamp at arrival; others: timestamp after the event  */
+  uint64_t seq;        /* PUSH: index of this learner's mini-batch, from 0                      */
+  uint64_t tick;       /* simulated arrival time (timed mode) or global push count (rounds)     */
+} rudra_event;
+
+/* mode: RUDRA_SCHED_*; hardsync requires n == 1.  lognormal_sigma: spread of ln(compute time)
+ * in timed mode.  downcast != 0: after every update the new weights are broadcast to all
+ * learners' receive buffers (Section 3.3), so per-learner pulls become inquiry skips.
+ * Returns NULL on invalid arguments. */
+rudra_sched* rudra_sched_create(uint32_t lambda, uint32_t n, int mode, uint64_t seed,
+                                double lognormal_sigma, int downcast);
+void rudra_sched_destroy(rudra_sched* s);
+/* Writes the next count events to out; returns count, or RUDRA_E_INVAL. */
+int64_t rudra_sched_next(rudra_sched* s, rudra_event* out, uint64_t count);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RUDRA_PS_H */

@@ -1,0 +1,441 @@
+// Host side of the parameter server: the message queue, the integer bookkeeping of Section 3.1
+// (scalar timestamp, staleness, vector clock, Eq. 2), the step-size table of Eq. 5 / Eq. 6 and
+// the launches.  All floating-point work on the model happens in the kernels of update.cu and
+// snapshot.cu; nothing here touches a weight.
+#include <cmath>
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <new>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "../../include/rudra_ps.h"
+#include "kernels.cuh"
+
+namespace {
+
+thread_local char g_error[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_error, sizeof(g_error), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+  return fail(RUDRA_E_CUDA, "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
+}
+
+constexpr uint32_t kMagic = 0x52554452u;   // "RUDR"
+constexpr uintptr_t kAlignMask = 31;       // 256-bit vector accesses
+
+bool aligned(const void* p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & kAlignMask) == 0; }
+
+struct Pending {
+  const void* grad;
+  uint64_t pulled_ts;
+  int slot;   // staging slot that holds the data, or -1 for a borrowed caller buffer
+};
+
+// Makes the handle's device current for the duration of a call.
+class DeviceScope {
+ public:
+  explicit DeviceScope(int device) : prev_(-1), ok_(true) {
+    if (cudaGetDevice(&prev_) != cudaSuccess) { ok_ = false; return; }
+    if (prev_ != device) { ok_ = cudaSetDevice(device) == cudaSuccess; switched_ = ok_; }
+  }
+  ~DeviceScope() { if (switched_) cudaSetDevice(prev_); }
+  bool ok() const { return ok_; }
+ private:
+  int prev_;
+  bool ok_;
+  bool switched_ = false;
+};
+
+}  // namespace
+
+struct rudra_ps {
+  uint32_t magic = kMagic;
+  uint64_t N = 0;
+  uint32_t lambda = 0, n = 0, c = 0;
+  float alpha0 = 0.f, momentum = 0.f, wd = 0.f, eps = 1e-8f;
+  int gtype = RUDRA_GRAD_F32, policy = RUDRA_LR_PAPER_N, optim = RUDRA_OPTIM_MOMENTUM_SGD;
+  int device = 0;
+  rudra::LaunchShape shape{1, 0};
+  cudaStream_t stream = nullptr;
+  float* theta = nullptr;
+  float* state = nullptr;
+  uint64_t ts = 0;
+  std::deque<Pending> queue;
+  std::vector<void*> slots;        // staging buffers for gradients pushed from host memory
+  std::vector<int> free_slots;
+  bool has_clock = false;
+  std::vector<uint64_t> clock;
+  std::vector<uint32_t> sigma;
+  std::vector<float> scale;
+  double avg_sigma = 0.0;
+  uint64_t counters[6] = {0, 0, 0, 0, 0, 0};
+
+  size_t grad_bytes() const { return (size_t)N * (gtype == RUDRA_GRAD_BF16 ? 2u : 4u); }
+};
+
+namespace {
+
+bool valid(const rudra_ps* ps) { return ps != nullptr && ps->magic == kMagic; }
+
+void release_queue(rudra_ps* ps) {
+  for (const Pending& e : ps->queue)
+    if (e.slot >= 0) ps->free_slots.push_back(e.slot);
+  ps->queue.clear();
+}
+
+int free_staging(rudra_ps* ps) {
+  cudaError_t e = cudaStreamSynchronize(ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  for (void* s : ps->slots) cudaFree(s);
+  ps->slots.clear();
+  ps->free_slots.clear();
+  return 0;
+}
+
+int64_t enqueue(rudra_ps* ps, const void* grad, uint64_t pulled_ts, int slot) {
+  ps->queue.push_back(Pending{grad, pulled_ts, slot});
+  ps->counters[0] += 1;
+  return (int64_t)ps->queue.size();
+}
+
+int check_push(rudra_ps* ps, uint64_t pulled_ts) {
+  // a learner cannot have pulled weights that do not exist yet: staleness is never negative
+  if (pulled_ts > ps->ts)
+    return fail(RUDRA_E_BAD_TS, "pulled_ts %llu is ahead of the server timestamp %llu",
+                (unsigned long long)pulled_ts, (unsigned long long)ps->ts);
+  if (ps->queue.size() >= RUDRA_QUEUE_CAP) return fail(RUDRA_E_QUEUE_FULL, "%d gradients already queued", RUDRA_QUEUE_CAP);
+  return 0;
+}
+
+// Group close (Section 3.1, Eq. 2) and the step-size table (Eq. 5's 1/c times the rate of Eq. 6
+// or one of its two variants).  Integers first, then one rounding to fp32 per table entry.
+void close_group(rudra_ps* ps, rudra::UpdateParams& p) {
+  const uint32_t c = ps->c;
+  ps->clock.resize(c);
+  ps->sigma.resize(c);
+  ps->scale.resize(c);
+  uint64_t sum_sigma = 0, sum_pulled = 0;
+  for (uint32_t l = 0; l < c; ++l) {
+    const Pending& e = ps->queue[l];
+    ps->clock[l] = e.pulled_ts;
+    ps->sigma[l] = (uint32_t)(ps->ts - e.pulled_ts);
+    sum_sigma += ps->sigma[l];
+    sum_pulled += e.pulled_ts;
+    p.grad[l] = e.grad;
+  }
+  ps->avg_sigma = (double)ps->ts - (double)sum_pulled / (double)c;
+  double sum_scale = 0.0;
+  for (uint32_t l = 0; l < c; ++l) {
+    double divisor;
+    switch (ps->policy) {
+      case RUDRA_LR_PER_GRADIENT: divisor = (double)(ps->sigma[l] > 1 ? ps->sigma[l] : 1u) * (double)c; break;
+      case RUDRA_LR_GROUP_MEAN:   divisor = (double)(sum_sigma > c ? sum_sigma : (uint64_t)c); break;
+      default:                    divisor = (double)ps->n * (double)c; break;
+    }
+    ps->scale[l] = (float)((double)ps->alpha0 / divisor);
+    sum_scale += (double)ps->scale[l];
+  }
+  const float abar = (float)sum_scale;
+  for (uint32_t l = 0; l < c; ++l)
+    p.scale[l] = ps->optim == RUDRA_OPTIM_ADAGRAD ? (float)((double)ps->scale[l] / (double)abar) : ps->scale[l];
+  p.theta = ps->theta;
+  p.state = ps->state;
+  p.n = ps->N;
+  p.c = c;
+  p.momentum = ps->momentum;
+  p.awd = (float)((double)abar * (double)ps->wd);
+  p.abar = abar;
+  p.wd = ps->wd;
+  p.eps = ps->eps;
+  ps->has_clock = true;
+}
+
+int do_step(rudra_ps* ps, float* const* dsts, uint32_t k) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (k > RUDRA_MAX_DSTS) return fail(RUDRA_E_INVAL, "k = %u exceeds RUDRA_MAX_DSTS", k);
+  if (k && !dsts) return fail(RUDRA_E_INVAL, "null destination list");
+  for (uint32_t d = 0; d < k; ++d)
+    if (!aligned(dsts[d])) return fail(RUDRA_E_INVAL, "destination %u is null or not 32-byte aligned", d);
+  if (ps->queue.size() < ps->c) return 0;   // group still open: nothing changes
+  DeviceScope dev(ps->device);
+  if (!dev.ok()) return fail(RUDRA_E_CUDA, "cannot select device %d", ps->device);
+  rudra::UpdateParams p;
+  close_group(ps, p);
+  p.ndst = k;
+  for (uint32_t d = 0; d < k; ++d) p.dst[d] = dsts[d];
+  cudaError_t e = rudra::launch_update(p, ps->gtype == RUDRA_GRAD_BF16 ? rudra::kBF16 : rudra::kF32,
+                                       ps->optim == RUDRA_OPTIM_ADAGRAD ? rudra::kAdagrad : rudra::kMomentumSgd,
+                                       ps->shape, ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "update kernel launch");
+  for (uint32_t l = 0; l < ps->c; ++l) {
+    if (ps->queue.front().slot >= 0) ps->free_slots.push_back(ps->queue.front().slot);
+    ps->queue.pop_front();
+  }
+  ps->ts += 1;   // exactly one increment per weight update
+  ps->counters[1] += 1;
+  ps->counters[2] += k;
+  ps->counters[3] += 1;
+  return 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rudra_last_error(void) { return g_error; }
+
+rudra_ps* rudra_ps_create(uint64_t nparams, uint32_t lambda, uint32_t n, float alpha0, float momentum,
+                          float weight_decay) {
+  if (nparams == 0 || lambda == 0 || n == 0 || n > lambda) {
+    fail(RUDRA_E_INVAL, "need nparams > 0 and 1 <= n <= lambda (got nparams=%llu lambda=%u n=%u)",
+         (unsigned long long)nparams, lambda, n);
+    return nullptr;
+  }
+  if (lambda / n > RUDRA_MAX_GROUP) {
+    fail(RUDRA_E_INVAL, "c = floor(lambda/n) = %u exceeds RUDRA_MAX_GROUP = %d", lambda / n, RUDRA_MAX_GROUP);
+    return nullptr;
+  }
+  if (!std::isfinite(alpha0) || !std::isfinite(momentum) || !std::isfinite(weight_decay) || alpha0 < 0.f ||
+      momentum < 0.f || momentum >= 1.f || weight_decay < 0.f) {
+    fail(RUDRA_E_INVAL, "alpha0, momentum, weight_decay must be finite, non-negative, momentum < 1");
+    return nullptr;
+  }
+  rudra_ps* ps = new (std::nothrow) rudra_ps;
+  if (!ps) { fail(RUDRA_E_CUDA, "out of host memory"); return nullptr; }
+  ps->N = nparams; ps->lambda = lambda; ps->n = n; ps->c = lambda / n;
+  ps->alpha0 = alpha0; ps->momentum = momentum; ps->wd = weight_decay;
+  cudaError_t e = cudaGetDevice(&ps->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ps->shape.sm_count, cudaDevAttrMultiProcessorCount, ps->device);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ps->theta), nparams * sizeof(float));
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ps->state), nparams * sizeof(float));
+  if (e == cudaSuccess) e = cudaMemset(ps->theta, 0, nparams * sizeof(float));
+  if (e == cudaSuccess) e = cudaMemset(ps->state, 0, nparams * sizeof(float));
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    cuda_fail(e, "rudra_ps_create");
+    cudaFree(ps->theta);
+    cudaFree(ps->state);
+    ps->magic = 0;
+    delete ps;
+    return nullptr;
+  }
+  return ps;
+}
+
+void rudra_ps_destroy(rudra_ps* ps) {
+  if (!valid(ps)) return;
+  DeviceScope dev(ps->device);
+  cudaStreamSynchronize(ps->stream);
+  for (void* s : ps->slots) cudaFree(s);
+  cudaFree(ps->theta);
+  cudaFree(ps->state);
+  ps->magic = 0;
+  delete ps;
+}
+
+int rudra_ps_set_stream(rudra_ps* ps, void* cuda_stream) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  ps->stream = static_cast<cudaStream_t>(cuda_stream);
+  return 0;
+}
+
+int rudra_ps_set_option(rudra_ps* ps, int key, int64_t value) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!ps->queue.empty()) return fail(RUDRA_E_STATE, "options can only change while no gradient is queued");
+  DeviceScope dev(ps->device);
+  switch (key) {
+    case RUDRA_OPT_GRAD_DTYPE:
+      if (value != RUDRA_GRAD_F32 && value != RUDRA_GRAD_BF16) return fail(RUDRA_E_INVAL, "unknown gradient type %lld", (long long)value);
+      if ((int)value != ps->gtype) {
+        int r = free_staging(ps);   // staging buffers are sized for the gradient type
+        if (r < 0) return r;
+        ps->gtype = (int)value;
+      }
+      return 0;
+    case RUDRA_OPT_LR_POLICY:
+      if (value < RUDRA_LR_PAPER_N || value > RUDRA_LR_GROUP_MEAN) return fail(RUDRA_E_INVAL, "unknown learning-rate policy %lld", (long long)value);
+      ps->policy = (int)value;
+      return 0;
+    case RUDRA_OPT_OPTIMIZER:
+      if (value != RUDRA_OPTIM_MOMENTUM_SGD && value != RUDRA_OPTIM_ADAGRAD) return fail(RUDRA_E_INVAL, "unknown optimizer %lld", (long long)value);
+      if ((int)value != ps->optim) {
+        cudaError_t e = cudaMemsetAsync(ps->state, 0, ps->N * sizeof(float), ps->stream);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+        ps->optim = (int)value;
+      }
+      return 0;
+    default:
+      return fail(RUDRA_E_INVAL, "unknown option key %d", key);
+  }
+}
+
+int rudra_ps_set_alpha0(rudra_ps* ps, float alpha0) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!std::isfinite(alpha0) || alpha0 < 0.f) return fail(RUDRA_E_INVAL, "alpha0 must be finite and non-negative");
+  ps->alpha0 = alpha0;
+  return 0;
+}
+
+static int set_weights_common(rudra_ps* ps, const float* src, cudaMemcpyKind kind) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!src) return fail(RUDRA_E_INVAL, "null source");
+  DeviceScope dev(ps->device);
+  cudaError_t e = cudaMemcpyAsync(ps->theta, src, ps->N * sizeof(float), kind, ps->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ps->state, 0, ps->N * sizeof(float), ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "rudra_ps_set_weights");
+  if (kind == cudaMemcpyHostToDevice) ps->counters[4] += ps->N * sizeof(float);
+  release_queue(ps);
+  ps->ts = 0;
+  ps->has_clock = false;
+  return 0;
+}
+
+int rudra_ps_set_weights(rudra_ps* ps, const float* src_dev) {
+  return set_weights_common(ps, src_dev, cudaMemcpyDeviceToDevice);
+}
+
+int rudra_ps_set_weights_host(rudra_ps* ps, const float* src_host) {
+  return set_weights_common(ps, src_host, cudaMemcpyHostToDevice);
+}
+
+int64_t rudra_ps_push(rudra_ps* ps, const void* grad_dev, uint64_t pulled_ts) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!aligned(grad_dev)) return fail(RUDRA_E_INVAL, "gradient pointer is null or not 32-byte aligned");
+  if (int r = check_push(ps, pulled_ts)) return r;
+  return enqueue(ps, grad_dev, pulled_ts, -1);
+}
+
+int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_ts) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!grad_host) return fail(RUDRA_E_INVAL, "null gradient pointer");
+  if (int r = check_push(ps, pulled_ts)) return r;
+  DeviceScope dev(ps->device);
+  int slot;
+  if (!ps->free_slots.empty()) {
+    slot = ps->free_slots.back();
+    ps->free_slots.pop_back();
+  } else {
+    void* buf = nullptr;
+    cudaError_t e = cudaMalloc(&buf, ps->grad_bytes());
+    if (e != cudaSuccess) return cuda_fail(e, "staging buffer allocation");
+    ps->slots.push_back(buf);
+    slot = (int)ps->slots.size() - 1;
+  }
+  // Stream order makes re-use safe: the update that read this slot was enqueued before this copy.
+  cudaError_t e = cudaMemcpyAsync(ps->slots[slot], grad_host, ps->grad_bytes(), cudaMemcpyHostToDevice, ps->stream);
+  if (e != cudaSuccess) {
+    ps->free_slots.push_back(slot);
+    return cuda_fail(e, "gradient host-to-device copy");
+  }
+  ps->counters[4] += ps->grad_bytes();
+  return enqueue(ps, ps->slots[slot], pulled_ts, slot);
+}
+
+int rudra_ps_step(rudra_ps* ps) { return do_step(ps, nullptr, 0); }
+
+int rudra_ps_step_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) { return do_step(ps, dsts_dev, k); }
+
+int64_t rudra_ps_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (k == 0) return (int64_t)ps->ts;
+  if (k > RUDRA_MAX_DSTS) return fail(RUDRA_E_INVAL, "k = %u exceeds RUDRA_MAX_DSTS", k);
+  if (!dsts_dev) return fail(RUDRA_E_INVAL, "null destination list");
+  rudra::SnapshotParams p;
+  for (uint32_t d = 0; d < k; ++d) {
+    if (!aligned(dsts_dev[d])) return fail(RUDRA_E_INVAL, "destination %u is null or not 32-byte aligned", d);
+    p.dst[d] = dsts_dev[d];
+  }
+  p.src = ps->theta;
+  p.n = ps->N;
+  p.ndst = k;
+  DeviceScope dev(ps->device);
+  cudaError_t e = rudra::launch_snapshot(p, ps->shape, ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "snapshot kernel launch");
+  ps->counters[2] += k;
+  ps->counters[3] += 1;
+  return (int64_t)ps->ts;
+}
+
+int64_t rudra_ps_pull(rudra_ps* ps, float* dst_dev) { return rudra_ps_pull_many(ps, &dst_dev, 1); }
+
+int64_t rudra_ps_pull_host(rudra_ps* ps, float* dst_host) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!dst_host) return fail(RUDRA_E_INVAL, "null destination");
+  DeviceScope dev(ps->device);
+  cudaError_t e = cudaMemcpyAsync(dst_host, ps->theta, ps->N * sizeof(float), cudaMemcpyDeviceToHost, ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "weights device-to-host copy");
+  ps->counters[2] += 1;
+  ps->counters[5] += ps->N * sizeof(float);
+  return (int64_t)ps->ts;
+}
+
+int64_t rudra_ps_timestamp(const rudra_ps* ps) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  return (int64_t)ps->ts;
+}
+
+int rudra_ps_last_clock(const rudra_ps* ps, uint64_t* pulled_ts_out, uint32_t* sigma_out, float* scale_out,
+                        double* avg_sigma_out) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!ps->has_clock) return 0;
+  for (uint32_t l = 0; l < ps->c; ++l) {
+    if (pulled_ts_out) pulled_ts_out[l] = ps->clock[l];
+    if (sigma_out) sigma_out[l] = ps->sigma[l];
+    if (scale_out) scale_out[l] = ps->scale[l];
+  }
+  if (avg_sigma_out) *avg_sigma_out = ps->avg_sigma;
+  return (int)ps->c;
+}
+
+int rudra_ps_export_state(rudra_ps* ps, float* theta_dst_dev, float* state_dst_dev) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  DeviceScope dev(ps->device);
+  cudaError_t e = cudaSuccess;
+  if (theta_dst_dev) e = cudaMemcpyAsync(theta_dst_dev, ps->theta, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
+  if (e == cudaSuccess && state_dst_dev)
+    e = cudaMemcpyAsync(state_dst_dev, ps->state, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "rudra_ps_export_state");
+  return 0;
+}
+
+int rudra_ps_import_state(rudra_ps* ps, const float* theta_src_dev, const float* state_src_dev, uint64_t ts) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  DeviceScope dev(ps->device);
+  cudaError_t e = cudaSuccess;
+  if (theta_src_dev) e = cudaMemcpyAsync(ps->theta, theta_src_dev, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
+  if (e == cudaSuccess && state_src_dev)
+    e = cudaMemcpyAsync(ps->state, state_src_dev, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "rudra_ps_import_state");
+  release_queue(ps);
+  ps->ts = ts;
+  ps->has_clock = false;
+  return 0;
+}
+
+int rudra_ps_sync(rudra_ps* ps) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  DeviceScope dev(ps->device);
+  cudaError_t e = cudaStreamSynchronize(ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  return 0;
+}
+
+int rudra_ps_counters(const rudra_ps* ps, uint64_t out[6]) {
+  if (!valid(ps) || !out) return fail(RUDRA_E_INVAL, "bad handle or null output");
+  std::memcpy(out, ps->counters, sizeof(ps->counters));
+  return 0;
+}
+
+}  // extern "C"

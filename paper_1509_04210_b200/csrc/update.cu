@@ -1,0 +1,223 @@
+// Fused sumGradients + applyUpdate kernel (Section 2; Eq. 5 with the rate of Eq. 6 folded into
+// per-gradient step sizes), sm_100a.
+//
+// The path is element-wise: weight k's new value depends on its own old value, its own state and
+// the c gradient values at index k.  So there is no reduction across threads, no shared memory
+// and no atomics; the kernel's only job is to keep enough bytes in flight to saturate HBM3e and
+// to touch every byte exactly once: c gradient reads, one read and one write of the weights and
+// of the state vector, and (optionally) ndst writes of the new weights into learner buffers.
+//
+// A thread works on units of 8 consecutive weights.  fp32 vectors move with 256-bit global loads
+// and stores (ld/st.global.v8.f32, new with sm_100), bf16 gradients with 128-bit loads, so a
+// warp instruction covers 1 KB (fp32) or 512 B (bf16) of contiguous memory.  Gradients are read
+// once and never again: they are loaded with an evict-first L2 policy and bypass L1, which leaves
+// L2 to the weights and state when the model is small enough to stay resident.
+#include <cuda_bf16.h>
+
+#include "kernels.cuh"
+
+namespace rudra {
+namespace {
+
+constexpr int kUnit = 8;   // weights per thread per unit
+
+struct alignas(32) F8 { float v[kUnit]; };
+
+__device__ __forceinline__ F8 ld8(const float* p) {
+  F8 r;
+  asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
+               : "l"(p));
+  return r;
+}
+
+__device__ __forceinline__ void st8(float* p, const F8& r) {
+  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
+               : "memory");
+}
+
+// One unit of one gradient stream, as loaded (fp32: 8 floats; bf16: 8 halves in 4 words).
+template <typename G> struct GradUnit;
+template <> struct GradUnit<float> {
+  F8 raw;
+  __device__ __forceinline__ void load(const void* base, uint64_t unit) {
+    const float* p = static_cast<const float*>(base) + unit * kUnit;
+    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(raw.v[0]), "=f"(raw.v[1]), "=f"(raw.v[2]), "=f"(raw.v[3]), "=f"(raw.v[4]), "=f"(raw.v[5]), "=f"(raw.v[6]), "=f"(raw.v[7])
+                 : "l"(p));
+  }
+  __device__ __forceinline__ void zero() {
+#pragma unroll
+    for (int e = 0; e < kUnit; ++e) raw.v[e] = 0.f;
+  }
+  __device__ __forceinline__ float get(int e) const { return raw.v[e]; }
+  static __device__ __forceinline__ float scalar(const void* base, uint64_t k) { return static_cast<const float*>(base)[k]; }
+};
+template <> struct GradUnit<__nv_bfloat16> {
+  uint4 raw;
+  __device__ __forceinline__ void load(const void* base, uint64_t unit) {
+    raw = __ldcs(static_cast<const uint4*>(base) + unit);
+  }
+  __device__ __forceinline__ void zero() { raw = make_uint4(0u, 0u, 0u, 0u); }
+  // bf16 is the upper half of an fp32: widening is a shift, exact.
+  __device__ __forceinline__ float get(int e) const {
+    const uint32_t w = e < 2 ? raw.x : e < 4 ? raw.y : e < 6 ? raw.z : raw.w;
+    return __uint_as_float((e & 1) ? (w & 0xFFFF0000u) : (w << 16));
+  }
+  static __device__ __forceinline__ float scalar(const void* base, uint64_t k) {
+    return __uint_as_float((uint32_t)static_cast<const uint16_t*>(base)[k] << 16);
+  }
+};
+
+// acc += s_l * g_l for K gradient streams starting at table entry l0: all K * U loads are issued
+// before the first use.
+template <typename G, int K, int U, int THREADS, bool GUARD>
+__device__ __forceinline__ void accumulate(const UpdateParams& p, uint32_t l0, uint64_t unit0, uint64_t nunits,
+                                           float (&acc)[U][kUnit]) {
+  GradUnit<G> g[K][U];
+#pragma unroll
+  for (int l = 0; l < K; ++l) {
+    const void* base = p.grad[l0 + l];
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+      const uint64_t u = unit0 + (uint64_t)j * THREADS;
+      if (!GUARD || u < nunits) g[l][j].load(base, u); else g[l][j].zero();
+    }
+  }
+#pragma unroll
+  for (int l = 0; l < K; ++l) {
+    const float s = p.scale[l0 + l];
+#pragma unroll
+    for (int j = 0; j < U; ++j)
+#pragma unroll
+      for (int e = 0; e < kUnit; ++e) acc[j][e] = fmaf(s, g[l][j].get(e), acc[j][e]);
+  }
+}
+
+// The per-weight rule.  Momentum SGD: u = acc + (sum s) wd theta; v' = m v + u; theta' = theta - v'.
+// AdaGrad: g = acc + wd theta (acc already the weighted mean gradient); h' = h + g^2;
+// theta' = theta - (sum s) g / (sqrt(h') + eps).
+template <int OPT, bool STATE>
+__device__ __forceinline__ void apply(const UpdateParams& p, float acc, float& theta, float& state) {
+  if (OPT == kMomentumSgd) {
+    const float u = fmaf(p.awd, theta, acc);
+    const float v = STATE ? fmaf(p.momentum, state, u) : u;
+    theta = theta - v;
+    state = v;
+  } else {
+    const float g = fmaf(p.wd, theta, acc);
+    const float h = fmaf(g, g, state);
+    theta = theta - __fdiv_rn(p.abar * g, __fsqrt_rn(h) + p.eps);
+    state = h;
+  }
+}
+
+template <typename G, int OPT, bool STATE, int KMAX, int U, int THREADS, bool GUARD>
+__device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t unit0, uint64_t nunits) {
+  F8 th[U], st[U];
+  float acc[U][kUnit];
+#pragma unroll
+  for (int j = 0; j < U; ++j) {
+    const uint64_t u = unit0 + (uint64_t)j * THREADS;
+    if (!GUARD || u < nunits) {
+      th[j] = ld8(p.theta + u * kUnit);
+      if (STATE) st[j] = ld8(p.state + u * kUnit);
+    }
+#pragma unroll
+    for (int e = 0; e < kUnit; ++e) acc[j][e] = 0.f;
+  }
+  uint32_t l = 0;
+  for (; l + KMAX <= p.c; l += KMAX) accumulate<G, KMAX, U, THREADS, GUARD>(p, l, unit0, nunits, acc);
+  switch (p.c - l) {   // uniform across the grid
+    case 7: if (KMAX > 7) accumulate<G, 7, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+    case 6: if (KMAX > 6) accumulate<G, 6, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+    case 5: if (KMAX > 5) accumulate<G, 5, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+    case 4: if (KMAX > 4) accumulate<G, 4, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+    case 3: if (KMAX > 3) accumulate<G, 3, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+    case 2: if (KMAX > 2) accumulate<G, 2, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+    case 1: accumulate<G, 1, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+    default: break;
+  }
+#pragma unroll
+  for (int j = 0; j < U; ++j) {
+    const uint64_t u = unit0 + (uint64_t)j * THREADS;
+    if (!GUARD || u < nunits) {
+#pragma unroll
+      for (int e = 0; e < kUnit; ++e) {
+        float s = STATE ? st[j].v[e] : 0.f;
+        apply<OPT, STATE>(p, acc[j][e], th[j].v[e], s);
+        if (STATE) st[j].v[e] = s;
+      }
+      st8(p.theta + u * kUnit, th[j]);
+      if (STATE) st8(p.state + u * kUnit, st[j]);
+      for (uint32_t d = 0; d < p.ndst; ++d) st8(p.dst[d] + u * kUnit, th[j]);
+    }
+  }
+}
+
+// Grid-stride over tiles of THREADS * U units; the last, ragged tile takes the guarded path and
+// the n % 8 trailing weights are done one by one by the first block.
+template <typename G, int OPT, bool STATE, int KMAX, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS) update_kernel(const __grid_constant__ UpdateParams p) {
+  const uint64_t nunits = p.n / kUnit;
+  constexpr uint64_t kTile = (uint64_t)THREADS * U;
+  const uint64_t full_tiles = nunits / kTile;
+  for (uint64_t tile = blockIdx.x; tile < full_tiles; tile += gridDim.x)
+    process_tile<G, OPT, STATE, KMAX, U, THREADS, false>(p, tile * kTile + threadIdx.x, nunits);
+  if (full_tiles * kTile < nunits && blockIdx.x == full_tiles % gridDim.x)
+    process_tile<G, OPT, STATE, KMAX, U, THREADS, true>(p, full_tiles * kTile + threadIdx.x, nunits);
+  const uint64_t k = nunits * kUnit + threadIdx.x;
+  if (blockIdx.x == 0 && k < p.n) {
+    float acc = 0.f;
+    for (uint32_t l = 0; l < p.c; ++l) acc = fmaf(p.scale[l], GradUnit<G>::scalar(p.grad[l], k), acc);
+    float th = p.theta[k];
+    float s = STATE ? p.state[k] : 0.f;
+    apply<OPT, STATE>(p, acc, th, s);
+    p.theta[k] = th;
+    if (STATE) p.state[k] = s;
+    for (uint32_t d = 0; d < p.ndst; ++d) p.dst[d][k] = th;
+  }
+}
+
+template <typename G, int OPT, bool STATE, int KMAX, int U, int THREADS>
+cudaError_t launch_one(const UpdateParams& p, const LaunchShape& shape, cudaStream_t stream) {
+  auto kern = update_kernel<G, OPT, STATE, KMAX, U, THREADS>;
+  static int cached_blocks_per_sm = 0;   // per instantiation; the occupancy of a kernel is fixed
+  int per_sm = shape.blocks_per_sm;
+  if (per_sm <= 0) {
+    if (cached_blocks_per_sm == 0) {
+      int b = 0;
+      cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kern, THREADS, 0);
+      if (e != cudaSuccess) return e;
+      cached_blocks_per_sm = b > 0 ? b : 1;
+    }
+    per_sm = cached_blocks_per_sm;
+  }
+  const uint64_t nunits = p.n / kUnit;
+  const uint64_t tiles = (nunits + (uint64_t)THREADS * U - 1) / ((uint64_t)THREADS * U);
+  uint64_t grid = (uint64_t)shape.sm_count * (uint64_t)per_sm;   // a whole number of waves
+  if (tiles < grid) grid = tiles;
+  if (grid == 0) grid = 1;                                        // n < 8: only the scalar tail
+  kern<<<(unsigned)grid, THREADS, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename G, int KMAX, int U, int THREADS>
+cudaError_t launch_typed(const UpdateParams& p, Optim optim, const LaunchShape& shape, cudaStream_t stream) {
+  if (optim == kAdagrad) return launch_one<G, kAdagrad, true, KMAX, U, THREADS>(p, shape, stream);
+  if (p.momentum != 0.f) return launch_one<G, kMomentumSgd, true, KMAX, U, THREADS>(p, shape, stream);
+  return launch_one<G, kMomentumSgd, false, KMAX, U, THREADS>(p, shape, stream);   // no velocity kept
+}
+
+}  // namespace
+
+cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, const LaunchShape& shape,
+                          cudaStream_t stream) {
+  if (gtype == kBF16) return launch_typed<__nv_bfloat16, 8, 1, 256>(p, optim, shape, stream);
+  // fp32: with few gradient streams a thread carries two units to keep enough loads in flight
+  if (p.c <= 2) return launch_typed<float, 4, 2, 256>(p, optim, shape, stream);
+  return launch_typed<float, 4, 1, 256>(p, optim, shape, stream);
+}
+
+}  // namespace rudra
