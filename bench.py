@@ -245,8 +245,9 @@ def run_ours(args, w):
     N = w.nparams
     seed = synth.MASTER_SEED + rank
     stream = torch.cuda.Stream()
-    bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype, seed) for l in range(w.lam)]
-    nslots = w.lam
+    nbufs = min(w.lam, args.buffers) if args.buffers else w.lam
+    bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype, seed) for l in range(nbufs)]
+    nslots = nbufs
     slots = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(nslots)]
     ps = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
     ps.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
@@ -258,7 +259,7 @@ def run_ours(args, w):
     def run_window(win, ev_pairs=None):
         for kind, learner, pulled_ts, ts in win:
             if kind == rb.EV_PUSH:
-                ps.push(bufs[learner], pulled_ts)
+                ps.push(bufs[learner % nbufs], pulled_ts)
             elif kind == rb.EV_STEP:
                 if ev_pairs is not None:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -269,7 +270,7 @@ def run_ours(args, w):
                 else:
                     ps.step()
             elif kind == rb.EV_PULL:
-                ps.pull(slots[learner])
+                ps.pull(slots[learner % nslots])
             elif kind == rb.EV_BROADCAST:
                 ps.pull_many(slots)
 
@@ -293,50 +294,52 @@ def run_ours(args, w):
     launches = c1["launches"] - c0["launches"]
     pulls = c1["pulls"] - c0["pulls"]
 
-    # end to end through the C interface with host buffers: gradients travel host -> device inside
-    # the timed region and every pulled copy of the weights travels device -> host
-    e2e_steps = min(args.steps, 16 if N > (1 << 24) else 200)
-    nhost = min(w.lam, 8)
-    hg = []
-    for l in range(nhost):
-        t = torch.empty(N, dtype=bufs[0].dtype).pin_memory()
-        t.copy_(bufs[l])
-        hg.append(t)
-    hdst = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(2)]
-    torch.cuda.synchronize()
-    ps2 = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
-    ps2.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
-    ps2.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
-    ps2.sync()
-    ps2.set_stream(stream)
+    e2e_ms, e2e_steps, h0, h1 = float('nan'), 0, None, None
+    if not args.kernel_only:
+        # end to end through the C interface with host buffers: gradients travel host -> device inside
+        # the timed region and every pulled copy of the weights travels device -> host
+        e2e_steps = min(args.steps, 16 if N > (1 << 24) else 200)
+        nhost = min(nbufs, 8)
+        hg = []
+        for l in range(nhost):
+            t = torch.empty(N, dtype=bufs[0].dtype).pin_memory()
+            t.copy_(bufs[l])
+            hg.append(t)
+        hdst = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(2)]
+        torch.cuda.synchronize()
+        ps2 = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
+        ps2.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
+        ps2.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
+        ps2.sync()
+        ps2.set_stream(stream)
 
-    def run_window_host(win):
-        k = 0
-        for kind, learner, pulled_ts, ts in win:
-            if kind == rb.EV_PUSH:
-                ps2.push_host(hg[learner % nhost], pulled_ts)
-            elif kind == rb.EV_STEP:
-                ps2.step()
-            elif kind == rb.EV_PULL:
-                ps2.pull_host(hdst[k % 2])
-                k += 1
-            elif kind == rb.EV_BROADCAST:
-                ps2.pull_host(hdst[0])   # one copy leaves the device; learners on the host share it
+        def run_window_host(win):
+            k = 0
+            for kind, learner, pulled_ts, ts in win:
+                if kind == rb.EV_PUSH:
+                    ps2.push_host(hg[learner % nhost], pulled_ts)
+                elif kind == rb.EV_STEP:
+                    ps2.step()
+                elif kind == rb.EV_PULL:
+                    ps2.pull_host(hdst[k % 2])
+                    k += 1
+                elif kind == rb.EV_BROADCAST:
+                    ps2.pull_host(hdst[0])   # one copy leaves the device; learners on the host share it
 
-    e2e_warm = min(args.warmup, 3)
-    for win in windows[:e2e_warm]:
-        run_window_host(win)
-    barrier()
-    h0 = ps2.counters()
-    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s2.record(stream)
-    for win in windows[e2e_warm: e2e_warm + e2e_steps]:
-        run_window_host(win)
-    e2.record(stream)
-    barrier()
-    h1 = ps2.counters()
-    e2e_ms = s2.elapsed_time(e2)
-    ps2.close()
+        e2e_warm = min(args.warmup, 3)
+        for win in windows[:e2e_warm]:
+            run_window_host(win)
+        barrier()
+        h0 = ps2.counters()
+        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s2.record(stream)
+        for win in windows[e2e_warm: e2e_warm + e2e_steps]:
+            run_window_host(win)
+        e2.record(stream)
+        barrier()
+        h1 = ps2.counters()
+        e2e_ms = s2.elapsed_time(e2)
+        ps2.close()
 
     times = torch.tensor([ms, e2e_ms, upd_ms], dtype=torch.float64, device="cuda")
     if world > 1:
@@ -360,7 +363,7 @@ def run_ours(args, w):
             "update_kernel_updates_per_sec": 1e3 / upd_ms,
             "gpu_launches": launches,
             "clocks": clocks,
-            "e2e": {
+            "e2e": None if args.kernel_only else {
                 "value": world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": (h1["h2d_bytes"] - h0["h2d_bytes"]) // e2e_steps,
                 "d2h_bytes_per_step": (h1["d2h_bytes"] - h0["d2h_bytes"]) // e2e_steps,
@@ -373,7 +376,7 @@ def run_ours(args, w):
                 "traffic": None,
             },
         }
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and not args.kernel_only:
             from oracle import rudra_oracle as ora
 
             ora.build()
@@ -401,9 +404,19 @@ def main():
     ap.add_argument("--workload", default="imagenet", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="device-resident timed region only: no end-to-end leg, no CPU baseline (profiler captures)")
+    ap.add_argument("--nparams", type=int, default=0,
+                    help="override the vector length (small cases for profiler captures; not a bench line)")
+    ap.add_argument("--buffers", type=int, default=0,
+                    help="distinct gradient buffers and learner slots (default: one per learner)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     w = synth.WORKLOADS[args.workload]
+    if args.nparams:
+        import dataclasses
+
+        w = dataclasses.replace(w, name=w.name + "@%d" % args.nparams, nparams=args.nparams)
     if args.impl == "reference":
         run_reference(args, w)
     else:
