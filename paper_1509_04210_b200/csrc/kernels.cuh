@@ -29,6 +29,7 @@ struct UpdateParams {
   float abar;                    // AdaGrad: sum(s), the group's learning rate
   float wd;                      // AdaGrad: weight decay
   float eps;                     // AdaGrad: denominator floor
+  uint32_t reverse;              // sweep the vector from the end (alternates launch to launch)
 };
 
 struct SnapshotParams {
@@ -36,18 +37,13 @@ struct SnapshotParams {
   const float* src;
   uint64_t n;
   uint32_t ndst;
-};
-
-struct LaunchShape {
-  int sm_count;          // multiprocessors of the device
-  int blocks_per_sm;     // 0 = let the occupancy calculator decide
+  uint32_t reverse;
 };
 
 // Enqueue one fused update (and ndst snapshot writes) on stream.  Returns the CUDA status of the launch.
-cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, const LaunchShape& shape,
-                          cudaStream_t stream);
+cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, cudaStream_t stream);
 
 // Enqueue one 1 -> ndst copy of the weights.
-cudaError_t launch_snapshot(const SnapshotParams& p, const LaunchShape& shape, cudaStream_t stream);
+cudaError_t launch_snapshot(const SnapshotParams& p, cudaStream_t stream);
 
 }  // namespace rudra

@@ -67,7 +67,7 @@ struct rudra_ps {
   float alpha0 = 0.f, momentum = 0.f, wd = 0.f, eps = 1e-8f;
   int gtype = RUDRA_GRAD_F32, policy = RUDRA_LR_PAPER_N, optim = RUDRA_OPTIM_MOMENTUM_SGD;
   int device = 0;
-  rudra::LaunchShape shape{1, 0};
+  uint32_t sweep = 0;              // launches so far: successive launches sweep in opposite directions
   cudaStream_t stream = nullptr;
   float* theta = nullptr;
   float* state = nullptr;
@@ -175,9 +175,10 @@ int do_step(rudra_ps* ps, float* const* dsts, uint32_t k) {
   close_group(ps, p);
   p.ndst = k;
   for (uint32_t d = 0; d < k; ++d) p.dst[d] = dsts[d];
+  p.reverse = ps->sweep++ & 1u;
   cudaError_t e = rudra::launch_update(p, ps->gtype == RUDRA_GRAD_BF16 ? rudra::kBF16 : rudra::kF32,
                                        ps->optim == RUDRA_OPTIM_ADAGRAD ? rudra::kAdagrad : rudra::kMomentumSgd,
-                                       ps->shape, ps->stream);
+                                       ps->stream);
   if (e != cudaSuccess) return cuda_fail(e, "update kernel launch");
   for (uint32_t l = 0; l < ps->c; ++l) {
     if (ps->queue.front().slot >= 0) ps->free_slots.push_back(ps->queue.front().slot);
@@ -217,7 +218,6 @@ rudra_ps* rudra_ps_create(uint64_t nparams, uint32_t lambda, uint32_t n, float a
   ps->N = nparams; ps->lambda = lambda; ps->n = n; ps->c = lambda / n;
   ps->alpha0 = alpha0; ps->momentum = momentum; ps->wd = weight_decay;
   cudaError_t e = cudaGetDevice(&ps->device);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ps->shape.sm_count, cudaDevAttrMultiProcessorCount, ps->device);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ps->theta), nparams * sizeof(float));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ps->state), nparams * sizeof(float));
   if (e == cudaSuccess) e = cudaMemset(ps->theta, 0, nparams * sizeof(float));
@@ -360,8 +360,9 @@ int64_t rudra_ps_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) {
   p.src = ps->theta;
   p.n = ps->N;
   p.ndst = k;
+  p.reverse = ps->sweep++ & 1u;
   DeviceScope dev(ps->device);
-  cudaError_t e = rudra::launch_snapshot(p, ps->shape, ps->stream);
+  cudaError_t e = rudra::launch_snapshot(p, ps->stream);
   if (e != cudaSuccess) return cuda_fail(e, "snapshot kernel launch");
   ps->counters[2] += k;
   ps->counters[3] += 1;

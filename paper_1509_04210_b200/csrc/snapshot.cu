@@ -29,53 +29,40 @@ template <int U, int THREADS>
 __global__ void __launch_bounds__(THREADS) snapshot_kernel(const __grid_constant__ SnapshotParams p) {
   const uint64_t nunits = p.n / kUnit;
   constexpr uint64_t kTile = (uint64_t)THREADS * U;
-  const uint64_t tiles = (nunits + kTile - 1) / kTile;
-  for (uint64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-    const uint64_t unit0 = tile * kTile + threadIdx.x;
-    F8 w[U];
+  const uint64_t tile = p.reverse ? (uint64_t)gridDim.x - 1 - blockIdx.x : (uint64_t)blockIdx.x;
+  const uint64_t unit0 = tile * kTile + threadIdx.x;
+  F8 w[U];
+#pragma unroll
+  for (int j = 0; j < U; ++j) {
+    const uint64_t u = unit0 + (uint64_t)j * THREADS;
+    if (u < nunits) w[j] = ld8(p.src + u * kUnit);
+  }
+  for (uint32_t d = 0; d < p.ndst; ++d) {
+    float* out = p.dst[d];
 #pragma unroll
     for (int j = 0; j < U; ++j) {
       const uint64_t u = unit0 + (uint64_t)j * THREADS;
-      if (u < nunits) w[j] = ld8(p.src + u * kUnit);
-    }
-    for (uint32_t d = 0; d < p.ndst; ++d) {
-      float* out = p.dst[d];
-#pragma unroll
-      for (int j = 0; j < U; ++j) {
-        const uint64_t u = unit0 + (uint64_t)j * THREADS;
-        if (u < nunits) st8(out + u * kUnit, w[j]);
-      }
+      if (u < nunits) st8(out + u * kUnit, w[j]);
     }
   }
   const uint64_t k = nunits * kUnit + threadIdx.x;   // the n % 8 trailing weights
-  if (blockIdx.x == 0 && k < p.n) {
-    const float w = p.src[k];
-    for (uint32_t d = 0; d < p.ndst; ++d) p.dst[d][k] = w;
+  if (tile == 0 && k < p.n) {
+    const float w1 = p.src[k];
+    for (uint32_t d = 0; d < p.ndst; ++d) p.dst[d][k] = w1;
   }
 }
 
 }  // namespace
 
-cudaError_t launch_snapshot(const SnapshotParams& p, const LaunchShape& shape, cudaStream_t stream) {
-  constexpr int U = 4, THREADS = 256;
-  auto kern = snapshot_kernel<U, THREADS>;
-  static int cached_blocks_per_sm = 0;
-  int per_sm = shape.blocks_per_sm;
-  if (per_sm <= 0) {
-    if (cached_blocks_per_sm == 0) {
-      int b = 0;
-      cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kern, THREADS, 0);
-      if (e != cudaSuccess) return e;
-      cached_blocks_per_sm = b > 0 ? b : 1;
-    }
-    per_sm = cached_blocks_per_sm;
-  }
+// One tile per block, blocks handed out in index order; direction alternates with the update
+// launches so the copy starts on the part of the weights that is still in L2.
+cudaError_t launch_snapshot(const SnapshotParams& p, cudaStream_t stream) {
+  constexpr int U = 2, THREADS = 256;
   const uint64_t nunits = p.n / kUnit;
-  const uint64_t tiles = (nunits + (uint64_t)THREADS * U - 1) / ((uint64_t)THREADS * U);
-  uint64_t grid = (uint64_t)shape.sm_count * (uint64_t)per_sm;
-  if (tiles < grid) grid = tiles;
-  if (grid == 0) grid = 1;
-  kern<<<(unsigned)grid, THREADS, 0, stream>>>(p);
+  uint64_t tiles = (nunits + (uint64_t)THREADS * U - 1) / ((uint64_t)THREADS * U);
+  if (tiles == 0) tiles = 1;
+  if (tiles > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
+  snapshot_kernel<U, THREADS><<<(unsigned)tiles, THREADS, 0, stream>>>(p);
   return cudaGetLastError();
 }
 
