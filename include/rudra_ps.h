@@ -161,6 +161,41 @@ int rudra_ps_counters(const rudra_ps* ps, uint64_t out[6]);
 /* Reason of the calling thread's most recent failure; static storage, never freed. */
 const char* rudra_last_error(void);
 
+/*
+ * rudra_ps_update_host_noalloc -- (The paper has no counterpart to this call; it exists for
+ * callers of this library that cannot allocate device memory.)
+ *
+ * Who needs it: a process that gave the whole GPU to its own memory pool at start-up, so that a
+ * later cudaMalloc fails or fragments the pool; or a loop that cannot tolerate the device-wide
+ * synchronisation an allocation causes.  rudra_ps_push_host stages host gradients in device
+ * buffers that it allocates on demand; this call does the same update with no allocation at all
+ * (no cudaMalloc, no cudaFree, no allocating library routine): the staging area is a fixed array
+ * of RUDRA_NOALLOC_MAX_FLOATS floats inside the library image, resident on every GPU that loads
+ * the library until the process exits.
+ *
+ * What it does: copies the c fp32 gradients grads_host[0..c-1] (host memory, nparams floats each)
+ * to the staging array on cuda_stream and enqueues the fused kernel of rudra_ps_step on
+ * caller-owned vectors:  acc = sum_l scales[l] * g_l[k];  u = acc + (sum_l scales[l]) *
+ * weight_decay * theta[k];  state[k] = momentum * state[k] + u;  theta[k] -= state[k].
+ * theta_dev / state_dev: device memory, nparams floats, 32-byte aligned, updated in place
+ * (state_dev may be NULL when momentum == 0).  scales: c step sizes in host memory (what
+ * rudra_ps_last_clock reports as scale_out).  The timestamp bookkeeping stays with the caller.
+ *
+ * Limits and hazards: c * round_up(nparams, 64) must not exceed RUDRA_NOALLOC_MAX_FLOATS, else
+ * RUDRA_E_INVAL with a message naming the limit.  Every call on a device shares the one array:
+ * calls whose device work may overlap (different streams or threads) race on it; calls ordered on
+ * one stream do not.  The array keeps the last call's gradients; nothing in it needs clearing
+ * because each call overwrites all it reads.  The first call on each device looks up the array's
+ * device address (cudaGetSymbolAddress, with that device current); make that first call before
+ * any stream capture begins.  Returns 0, or RUDRA_E_INVAL / RUDRA_E_CUDA with the reason in
+ * rudra_noalloc_last_error().
+ */
+#define RUDRA_NOALLOC_MAX_FLOATS (4u * 1024u * 1024u)
+int rudra_ps_update_host_noalloc(float* theta_dev, float* state_dev, uint64_t nparams,
+                                 const float* const* grads_host, const float* scales, uint32_t c,
+                                 float momentum, float weight_decay, void* cuda_stream);
+const char* rudra_noalloc_last_error(void);
+
 /* ------------------------------------------------------------------------------------------
  * Learner event model.  The paper's server handles incoming messages strictly one by one
  * (Section 3.2), which makes the arrival order the whole control; this host-only scheduler

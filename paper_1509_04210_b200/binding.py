@@ -77,6 +77,8 @@ def lib():
         "rudra_ps_sync": (C.c_int, [vp]),
         "rudra_ps_counters": (C.c_int, [vp, vp]),
         "rudra_last_error": (C.c_char_p, []),
+        "rudra_ps_update_host_noalloc": (C.c_int, [vp, vp, u64, vp, vp, u32, f32, f32, vp]),
+        "rudra_noalloc_last_error": (C.c_char_p, []),
         "rudra_sched_create": (vp, [u32, u32, C.c_int, u64, C.c_double, C.c_int]),
         "rudra_sched_destroy": (None, [vp]),
         "rudra_sched_next": (i64, [vp, vp, u64]),
@@ -115,6 +117,23 @@ def _ptr(x):
 def _ptr_array(xs):
     arr = (C.c_void_p * len(xs))(*[_ptr(x) for x in xs])
     return arr
+
+
+NOALLOC_MAX_FLOATS = 4 * 1024 * 1024
+
+
+def update_host_noalloc(theta_dev, state_dev, nparams, grads_host, scales, momentum, weight_decay, stream=None):
+    """rudra_ps_update_host_noalloc: one fused update from host gradients, staged in the library's
+    fixed device array instead of allocated buffers (for callers that must not allocate)."""
+    c = len(grads_host)
+    table = _ptr_array(grads_host)
+    sc = np.ascontiguousarray(scales, dtype=np.float32)
+    handle = stream.cuda_stream if hasattr(stream, "cuda_stream") else stream
+    code = lib().rudra_ps_update_host_noalloc(_ptr(theta_dev), _ptr(state_dev), int(nparams), table, sc.ctypes.data, c,
+                                              momentum, weight_decay, handle)
+    if code < 0:
+        raise RudraError(code, lib().rudra_noalloc_last_error().decode())
+    return code
 
 
 class Scheduler:
