@@ -53,30 +53,47 @@ EV_PUSH, EV_STEP, EV_PULL, EV_PULL_SKIP, EV_BROADCAST = 1, 2, 3, 4, 5
 
 
 def make_windows(w, count, seed=synth.MASTER_SEED, from_oracle=False):
-    """Event windows: a window runs from the first push of a group to the last pull before the
-    next group's first push.  The CUDA arm takes the events from the library's scheduler, the
-    reference arm from the oracle's."""
+    """Event windows (arrays of event records): a window runs from the first push of a group to
+    the last pull before the next group's first push.  The CUDA arm takes the events from the
+    library's scheduler, the reference arm from the oracle's."""
     if from_oracle:
         from oracle import rudra_oracle as ora
 
         osched = ora.OracleScheduler(w.lam, w.n, w.mode, seed, w.lognormal_sigma, w.downcast)
-        next_event = lambda: osched.run(1)[0]
+        more = lambda k: osched.run(k)
     else:
         from paper_1509_04210_b200 import binding as rb
 
         sched = rb.Scheduler(w.lam, w.n, w.mode, seed, w.lognormal_sigma, w.downcast)
-        next_event = lambda: sched.next(1)[0]
+        more = lambda k: sched.next(k)
     windows, cur, stepped = [], [], False
     while len(windows) < count:
-        ev = next_event()
-        kind = int(ev["kind"])
-        if kind == EV_PUSH and stepped:
-            windows.append(cur)
-            cur, stepped = [], False
-        cur.append((kind, int(ev["learner"]), int(ev["pulled_ts"]), int(ev["ts"])))
-        if kind == EV_STEP:
-            stepped = True
+        for ev in more(4096):
+            if ev["kind"] == EV_PUSH and stepped:
+                windows.append(np.array(cur, dtype=ev.dtype))
+                cur, stepped = [], False
+                if len(windows) == count:
+                    break
+            cur.append(ev)
+            if ev["kind"] == EV_STEP:
+                stepped = True
     return windows
+
+
+def default_window(w):
+    """Updates packed into one launch by default: the gradients lambda learners can have waiting at
+    once make n = lambda / c updates (every learner blocks on its push until the server has taken
+    it), capped by the launch tables (32 updates, 128 gradients)."""
+    return max(1, min(w.n, 32, 128 // w.c))
+
+
+def window_bytes_per_param(w, events):
+    """Algorithmic bytes per weight of one launch over these events: every gradient read once,
+    weights and state read and written once, one write per pulled copy."""
+    g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
+    pushes = int((events["kind"] == EV_STEP).sum()) * w.c
+    pulls = int((events["kind"] == EV_PULL).sum()) + w.lam * int((events["kind"] == EV_BROADCAST).sum())
+    return pushes * g + (16 if w.momentum != 0.0 else 8) + 4 * pulls
 
 
 class ClockSampler(threading.Thread):
@@ -157,7 +174,7 @@ def oracle_run(w, windows, nsample, grads_host, warmup=0, budget_s=None, max_win
     for win in windows:
         if done == 0:
             t0 = time.perf_counter()
-        for kind, learner, pulled_ts, ts in win:
+        for kind, learner, pulled_ts in zip(win["kind"].tolist(), win["learner"].tolist(), win["pulled_ts"].tolist()):
             if kind == ora.PUSH:
                 ps.push(grads_host[learner % len(grads_host)], pulled_ts)
             elif kind == ora.STEP:
@@ -212,8 +229,9 @@ def workload_config(w):
         "momentum": w.momentum, "weight_decay": w.weight_decay,
         "grad_dtype": "bf16" if w.grad_dtype == synth.GRAD_BF16 else "f32",
         "scheduler": {0: "hardsync", 1: "softsync_rounds", 2: "softsync_timed"}[w.mode],
-        "l2": "inputs larger than L2: one distinct gradient buffer per learner, %.2f GB touched per update window"
-              % ((update_bytes_per_param(w) + 8 * w.c) * w.nparams / 1e9),
+        "l2": ("inputs larger than L2 (one distinct %.0f MB gradient buffer per learner, %.0f MB of weights and state)"
+               % (w.nparams * (2 if w.grad_dtype == synth.GRAD_BF16 else 4) / 1e6, w.nparams * 8 / 1e6))
+              if w.nparams * 8 > 126e6 else "weights and state fit in L2: launch-bound workload, no HBM roofline claim",
         "parallelism": "replicas",
     }
 
@@ -226,9 +244,9 @@ def run_ours(args, w):
     import torch.distributed as dist
     from paper_1509_04210_b200 import binding as rb
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_1509_04210_b200 import replicas
+
+    rank, local_rank, world = replicas.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
     torch.cuda.set_device(local_rank)
@@ -243,7 +261,7 @@ def run_ours(args, w):
         torch.cuda.synchronize()
 
     N = w.nparams
-    seed = synth.MASTER_SEED + rank
+    seed = replicas.replica_seed(synth.MASTER_SEED, rank)
     stream = torch.cuda.Stream()
     nbufs = min(w.lam, args.buffers) if args.buffers else w.lam
     bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype, seed) for l in range(nbufs)]
@@ -255,42 +273,64 @@ def run_ours(args, w):
     ps.sync()
     ps.set_stream(stream)
     windows = make_windows(w, args.warmup + args.steps)
+    W = default_window(w) if args.window < 0 else args.window
+    gtable = rb.pointer_table([bufs[l % nbufs] for l in range(w.lam)])
+    stable = rb.pointer_table([slots[l % nslots] for l in range(w.lam)])
 
-    def run_window(win, ev_pairs=None):
-        for kind, learner, pulled_ts, ts in win:
-            if kind == rb.EV_PUSH:
+    def new_events():
+        return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def run_messages(win, timed):
+        """One message at a time through push / step / pull (--window 0)."""
+        for kind, learner, pulled_ts in zip(win["kind"].tolist(), win["learner"].tolist(), win["pulled_ts"].tolist()):
+            if kind == EV_PUSH:
                 ps.push(bufs[learner % nbufs], pulled_ts)
-            elif kind == rb.EV_STEP:
-                if ev_pairs is not None:
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record(stream)
-                    ps.step()
-                    e1.record(stream)
-                    ev_pairs.append((e0, e1))
-                else:
-                    ps.step()
-            elif kind == rb.EV_PULL:
+            elif kind == EV_STEP:
+                e0, e1 = new_events()
+                e0.record(stream)
+                ps.step()
+                e1.record(stream)
+                timed.append((e0, e1, update_bytes_per_param(w) * N))
+            elif kind == EV_PULL:
                 ps.pull(slots[learner % nslots])
-            elif kind == rb.EV_BROADCAST:
+            elif kind == EV_BROADCAST:
                 ps.pull_many(slots)
 
-    for win in windows[: args.warmup]:
-        run_window(win)
+    def run_backlog(chunk, timed):
+        """A backlog of W update windows through run_events: one launch when the tables allow."""
+        before = ps.counters()["launches"]
+        e0, e1 = new_events()
+        e0.record(stream)
+        ps.run_events(chunk, gtable, stable, W)
+        e1.record(stream)
+        if ps.counters()["launches"] == before + 1:
+            timed.append((e0, e1, window_bytes_per_param(w, chunk) * N))
+
+    def run_all(wins, timed):
+        if W == 0:
+            for win in wins:
+                run_messages(win, timed)
+        else:
+            for i in range(0, len(wins), W):
+                run_backlog(np.concatenate(wins[i:i + W]), timed)
+
+    run_all(windows[: args.warmup], [])
     barrier()
     sampler = ClockSampler(visible_gpu_index(local_rank))
     sampler.start()
     c0 = ps.counters()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    pairs = []
+    start, end = new_events()
+    timed = []
     start.record(stream)
-    for win in windows[args.warmup:]:
-        run_window(win, pairs)
+    run_all(windows[args.warmup:], timed)
     end.record(stream)
     barrier()
     clocks = sampler.stop()
     c1 = ps.counters()
     ms = start.elapsed_time(end)
-    upd_ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+    kern_ms = float(sum(a.elapsed_time(b) for a, b, _ in timed))
+    kern_bytes = float(sum(nb for _, _, nb in timed))
+    upd_ms = kern_ms / max(len(timed), 1)
     launches = c1["launches"] - c0["launches"]
     pulls = c1["pulls"] - c0["pulls"]
 
@@ -315,15 +355,15 @@ def run_ours(args, w):
 
         def run_window_host(win):
             k = 0
-            for kind, learner, pulled_ts, ts in win:
-                if kind == rb.EV_PUSH:
+            for kind, learner, pulled_ts in zip(win["kind"].tolist(), win["learner"].tolist(), win["pulled_ts"].tolist()):
+                if kind == EV_PUSH:
                     ps2.push_host(hg[learner % nhost], pulled_ts)
-                elif kind == rb.EV_STEP:
+                elif kind == EV_STEP:
                     ps2.step()
-                elif kind == rb.EV_PULL:
+                elif kind == EV_PULL:
                     ps2.pull_host(hdst[k % 2])
                     k += 1
-                elif kind == rb.EV_BROADCAST:
+                elif kind == EV_BROADCAST:
                     ps2.pull_host(hdst[0])   # one copy leaves the device; learners on the host share it
 
         e2e_warm = min(args.warmup, 3)
@@ -341,37 +381,44 @@ def run_ours(args, w):
         e2e_ms = s2.elapsed_time(e2)
         ps2.close()
 
-    times = torch.tensor([ms, e2e_ms, upd_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_ms, upd_ms = (float(x) for x in times.cpu())
+    ms, e2e_ms, upd_ms = replicas.max_over_ranks([ms, e2e_ms, upd_ms], device="cuda")
 
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
-        bpp = update_bytes_per_param(w)
-        upd_bytes = bpp * N
-        achieved = upd_bytes / (upd_ms * 1e-3) / 1e9
-        window_bytes = (upd_bytes * args.steps + 8 * N * pulls) / args.steps
-        value = world * args.steps / (ms * 1e-3)
+        g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
+        achieved = kern_bytes / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else float("nan")
+        # bytes the whole path must move per step: every gradient once, weights/state per launch, pulls
+        state_bytes = 16 if w.momentum != 0.0 else 8
+        if W == 0:
+            path_bytes = N * (args.steps * (w.c * g + state_bytes) + 8 * pulls)
+        else:
+            path_bytes = N * (args.steps * w.c * g + launches * state_bytes + 4 * pulls)
+        value = replicas.whole_job_rate(args.steps, world, ms)
+        cfg = workload_config(w)
+        cfg["window"] = W
+        cfg["window_note"] = ("messages handled one at a time (push / step / pull)" if W == 0 else
+                              "backlog of %d update windows per rudra_ps_run_events call" % W)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(w),
-            "hbm_gbs_whole_path": window_bytes / (ms / args.steps * 1e-3) / 1e9,
+            "config": cfg,
+            "hbm_gbs_whole_path": path_bytes / (ms * 1e-3) / 1e9,
+            "bytes_per_param_per_step": path_bytes / N / args.steps,
             "pulls_per_step": pulls / args.steps,
-            "update_kernel_updates_per_sec": 1e3 / upd_ms,
             "gpu_launches": launches,
             "clocks": clocks,
             "e2e": None if args.kernel_only else {
-                "value": world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                "value": replicas.whole_job_rate(e2e_steps, world, e2e_ms), "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": (h1["h2d_bytes"] - h0["h2d_bytes"]) // e2e_steps,
                 "d2h_bytes_per_step": (h1["d2h_bytes"] - h0["d2h_bytes"]) // e2e_steps,
             },
             "roofline": {
-                "kernel": "update_kernel (fused sumGradients + applyUpdate)", "bound": "hbm",
-                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_kind": "of %s" % peak_kind, "bytes_per_param": bpp, "avg_launch_us": upd_ms * 1e3,
+                "kernel": "update_kernel (fused sumGradients + applyUpdate%s)" % (
+                    "" if W == 0 else ", %d-update window with its pulls" % W),
+                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": "of %s" % peak_kind, "launches_timed": len(timed), "avg_launch_us": upd_ms * 1e3,
+                "bytes_per_launch": kern_bytes / max(len(timed), 1),
                 "frac_of_8TBs_datasheet": achieved / 8000.0,
                 "traffic": None,
             },
@@ -403,6 +450,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="imagenet", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--window", type=int, default=-1,
+                    help="update windows handed to the server per call: 0 = one message at a time, "
+                         "-1 = what lambda blocked learners can have waiting (n = lambda/c updates)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-only", action="store_true",
                     help="device-resident timed region only: no end-to-end leg, no CPU baseline (profiler captures)")

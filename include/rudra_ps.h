@@ -231,6 +231,29 @@ void rudra_sched_destroy(rudra_sched* s);
 /* Writes the next count events to out; returns count, or RUDRA_E_INVAL. */
 int64_t rudra_sched_next(rudra_sched* s, rudra_event* out, uint64_t count);
 
+/*
+ * rudra_ps_run_events -- handle a backlog of messages.  Section 3.2's server takes messages one at
+ * a time and Section 5.2 / 5.5 name the cost: with many learners and small mini-batches updates
+ * and pulls arrive faster than the server finishes them.  This call takes the waiting messages in
+ * arrival order (events[0..count-1], as rudra_sched_next produces them) and does exactly what
+ * rudra_ps_push / rudra_ps_step / rudra_ps_pull / rudra_ps_pull_many would do one by one -- same
+ * timestamps, same staleness, bit-identical weights, state and pulled copies -- but packs
+ * consecutive updates and the pulls between them into one launch: the weights and the state stay
+ * in registers across up to max_window updates (0 = as many as the launch tables hold: at most
+ * 32 updates, RUDRA_MAX_GROUP gradients and RUDRA_MAX_DSTS pull destinations per launch), every
+ * gradient is read once and every pull is a store.  Per weight a window of W updates with P pulls
+ * moves W*c*G + 16 + 4*P bytes instead of W*(c*G + 16) + 8*P.
+ *
+ * grads_dev[l] is learner l's gradient buffer (read by the update that consumes the push, as in
+ * rudra_ps_push), slots_dev[l] its weight buffer (written by its pulls and by broadcasts); both
+ * are host arrays of lambda device pointers; slots_dev may be NULL if no event pulls.  The events'
+ * ts fields are checked against the server's timestamp.  The whole batch is validated before
+ * anything is queued or launched: on a negative return nothing has changed.  Returns the number
+ * of updates performed.
+ */
+int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t count,
+                            const void* const* grads_dev, float* const* slots_dev, uint32_t max_window);
+
 #ifdef __cplusplus
 }
 #endif

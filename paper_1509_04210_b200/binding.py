@@ -82,6 +82,7 @@ def lib():
         "rudra_sched_create": (vp, [u32, u32, C.c_int, u64, C.c_double, C.c_int]),
         "rudra_sched_destroy": (None, [vp]),
         "rudra_sched_next": (i64, [vp, vp, u64]),
+        "rudra_ps_run_events": (i64, [vp, vp, u64, vp, vp, u32]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -117,6 +118,11 @@ def _ptr(x):
 def _ptr_array(xs):
     arr = (C.c_void_p * len(xs))(*[_ptr(x) for x in xs])
     return arr
+
+
+def pointer_table(xs):
+    """Host array of device addresses, reusable across calls."""
+    return _ptr_array(xs)
 
 
 NOALLOC_MAX_FLOATS = 4 * 1024 * 1024
@@ -208,6 +214,14 @@ class ParameterServer:
     def pull_many(self, dsts_dev):
         arr = _ptr_array(dsts_dev)
         return _check(lib().rudra_ps_pull_many(self._h, arr, len(dsts_dev)))
+
+    def run_events(self, events, grads_dev, slots_dev=None, max_window=0):
+        """events: array of EVENT_DTYPE; grads_dev / slots_dev: per-learner buffers (lists of tensors,
+        or pointer tables made with ``pointer_table``)."""
+        ev = np.ascontiguousarray(events, dtype=EVENT_DTYPE)
+        g = grads_dev if isinstance(grads_dev, C.Array) else _ptr_array(grads_dev)
+        sl = None if slots_dev is None else (slots_dev if isinstance(slots_dev, C.Array) else _ptr_array(slots_dev))
+        return _check(lib().rudra_ps_run_events(self._h, ev.ctypes.data, len(ev), g, sl, int(max_window)))
 
     def timestamp(self):
         return _check(lib().rudra_ps_timestamp(self._h))

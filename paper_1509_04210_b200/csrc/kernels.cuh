@@ -11,26 +11,34 @@ constexpr int kMaxDsts = 128;    // RUDRA_MAX_DSTS
 enum GradType : int { kF32 = 0, kBF16 = 1 };
 enum Optim : int { kMomentumSgd = 0, kAdagrad = 1 };
 
-// Everything one fused sumGradients + applyUpdate launch needs.  Passed by value as a
-// __grid_constant__ kernel parameter: the per-gradient pointers and step sizes form a small
-// table in the constant bank, read with uniform addresses, so an update costs one launch and no
-// other stream operation.
+constexpr int kMaxWindow = 32;   // most updates one launch can carry
+
+// Everything one launch of the fused kernel needs: a window of nupd consecutive updates (each
+// sumGradients + applyUpdate over c gradients) with the pulls that fall between them.  Passed by
+// value as a __grid_constant__ kernel parameter: the gradient pointers, step sizes and pull
+// destinations form a small table in the constant bank, read with uniform addresses, so a window
+// costs one launch and no other stream operation.  Update u uses grad[u*c .. u*c+c-1]; pull
+// destinations dst[dst_end[u] .. dst_end[u+1]-1] receive the weights after update u, and
+// dst[0 .. dst_end[0]-1] the weights as they were before the window.
 struct UpdateParams {
-  const void* grad[kMaxGroup];   // c gradient vectors, arrival order
-  float* dst[kMaxDsts];          // ndst learner buffers that receive the new weights
-  float scale[kMaxGroup];        // s_l (momentum SGD) or s_l / sum(s) (AdaGrad)
+  const void* grad[kMaxGroup];   // nupd * c gradient vectors, arrival order
+  float* dst[kMaxDsts];          // learner buffers, in the order the pulls arrived
+  float scale[kMaxGroup];        // s_l (momentum SGD) or s_l / sum(s) (AdaGrad), aligned with grad[]
+  float awd[kMaxWindow];         // per update, momentum SGD: sum(s) * weight_decay
+  float abar[kMaxWindow];        // per update, AdaGrad: sum(s), the group's learning rate
+  uint8_t dst_end[kMaxWindow + 1];
   float* theta;
   float* state;                  // velocity (momentum SGD) or sum of squared gradients (AdaGrad)
   uint64_t n;                    // number of weights
-  uint32_t c;
-  uint32_t ndst;
+  uint32_t c;                    // gradients per update
+  uint32_t nupd;                 // updates in this window (>= 1)
   float momentum;
-  float awd;                     // momentum SGD: sum(s) * weight_decay
-  float abar;                    // AdaGrad: sum(s), the group's learning rate
   float wd;                      // AdaGrad: weight decay
   float eps;                     // AdaGrad: denominator floor
   uint32_t reverse;              // sweep the vector from the end (alternates launch to launch)
 };
+static_assert(sizeof(UpdateParams) <= 4096, "kernel parameters are limited to 4 KB");
+static_assert(kMaxDsts <= 255 && kMaxGroup <= 255, "table indices are stored in bytes");
 
 struct SnapshotParams {
   float* dst[kMaxDsts];
@@ -40,7 +48,7 @@ struct SnapshotParams {
   uint32_t reverse;
 };
 
-// Enqueue one fused update (and ndst snapshot writes) on stream.  Returns the CUDA status of the launch.
+// Enqueue one window of fused updates (and their pulls) on stream.  Returns the CUDA status of the launch.
 cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, cudaStream_t stream);
 
 // Enqueue one 1 -> ndst copy of the weights.

@@ -104,10 +104,11 @@ int rudra_ps_update_host_noalloc(float* theta_dev, float* state_dev, uint64_t np
   p.state = state_dev;
   p.n = nparams;
   p.c = c;
-  p.ndst = 0;
+  p.nupd = 1;
+  p.dst_end[0] = p.dst_end[1] = 0;
   p.momentum = momentum;
-  p.awd = (float)((double)abar * (double)weight_decay);
-  p.abar = abar;
+  p.awd[0] = (float)((double)abar * (double)weight_decay);
+  p.abar[0] = abar;
   p.wd = weight_decay;
   p.eps = 0.f;
   p.reverse = 0;

@@ -119,10 +119,20 @@ int check_push(rudra_ps* ps, uint64_t pulled_ts) {
   return 0;
 }
 
+// A launch under construction: a window of consecutive updates and the pulls between them.
+struct Window {
+  rudra::UpdateParams p;
+  uint32_t nupd = 0, ndst = 0;
+  std::vector<int> used_slots;   // staging slots the window's gradients occupy
+};
+
 // Group close (Section 3.1, Eq. 2) and the step-size table (Eq. 5's 1/c times the rate of Eq. 6
-// or one of its two variants).  Integers first, then one rounding to fp32 per table entry.
-void close_group(rudra_ps* ps, rudra::UpdateParams& p) {
+// or one of its two variants) for the c oldest queued gradients, appended to the window as its
+// next update.  Integers first, then one rounding to fp32 per table entry.  Raises the timestamp.
+void append_update(rudra_ps* ps, Window& w) {
   const uint32_t c = ps->c;
+  rudra::UpdateParams& p = w.p;
+  const uint32_t base = w.nupd * c;
   ps->clock.resize(c);
   ps->sigma.resize(c);
   ps->scale.resize(c);
@@ -133,7 +143,8 @@ void close_group(rudra_ps* ps, rudra::UpdateParams& p) {
     ps->sigma[l] = (uint32_t)(ps->ts - e.pulled_ts);
     sum_sigma += ps->sigma[l];
     sum_pulled += e.pulled_ts;
-    p.grad[l] = e.grad;
+    p.grad[base + l] = e.grad;
+    if (e.slot >= 0) w.used_slots.push_back(e.slot);
   }
   ps->avg_sigma = (double)ps->ts - (double)sum_pulled / (double)c;
   double sum_scale = 0.0;
@@ -149,17 +160,55 @@ void close_group(rudra_ps* ps, rudra::UpdateParams& p) {
   }
   const float abar = (float)sum_scale;
   for (uint32_t l = 0; l < c; ++l)
-    p.scale[l] = ps->optim == RUDRA_OPTIM_ADAGRAD ? (float)((double)ps->scale[l] / (double)abar) : ps->scale[l];
-  p.theta = ps->theta;
-  p.state = ps->state;
-  p.n = ps->N;
-  p.c = c;
-  p.momentum = ps->momentum;
-  p.awd = (float)((double)abar * (double)ps->wd);
-  p.abar = abar;
-  p.wd = ps->wd;
-  p.eps = ps->eps;
+    p.scale[base + l] = ps->optim == RUDRA_OPTIM_ADAGRAD ? (float)((double)ps->scale[l] / (double)abar) : ps->scale[l];
+  p.awd[w.nupd] = (float)((double)abar * (double)ps->wd);
+  p.abar[w.nupd] = abar;
+  p.dst_end[w.nupd] = (uint8_t)w.ndst;   // pulls so far belong to the state before this update
+  w.nupd += 1;
   ps->has_clock = true;
+  for (uint32_t l = 0; l < c; ++l) ps->queue.pop_front();
+  ps->ts += 1;   // exactly one increment per weight update
+}
+
+bool window_has_room_for_update(const rudra_ps* ps, const Window& w, uint32_t max_updates) {
+  return w.nupd < max_updates && (w.nupd + 1) * ps->c <= (uint32_t)rudra::kMaxGroup;
+}
+
+// Enqueues the window: the fused kernel if it holds updates, a plain snapshot if it holds only pulls.
+int flush_window(rudra_ps* ps, Window& w) {
+  if (w.nupd == 0 && w.ndst == 0) return 0;
+  cudaError_t e;
+  if (w.nupd == 0) {
+    rudra::SnapshotParams sp;
+    for (uint32_t d = 0; d < w.ndst; ++d) sp.dst[d] = w.p.dst[d];
+    sp.src = ps->theta;
+    sp.n = ps->N;
+    sp.ndst = w.ndst;
+    sp.reverse = ps->sweep++ & 1u;
+    e = rudra::launch_snapshot(sp, ps->stream);
+  } else {
+    rudra::UpdateParams& p = w.p;
+    p.dst_end[w.nupd] = (uint8_t)w.ndst;
+    p.theta = ps->theta;
+    p.state = ps->state;
+    p.n = ps->N;
+    p.c = ps->c;
+    p.nupd = w.nupd;
+    p.momentum = ps->momentum;
+    p.wd = ps->wd;
+    p.eps = ps->eps;
+    p.reverse = ps->sweep++ & 1u;
+    e = rudra::launch_update(p, ps->gtype == RUDRA_GRAD_BF16 ? rudra::kBF16 : rudra::kF32,
+                             ps->optim == RUDRA_OPTIM_ADAGRAD ? rudra::kAdagrad : rudra::kMomentumSgd, ps->stream);
+  }
+  for (int slot : w.used_slots) ps->free_slots.push_back(slot);   // stream order protects re-use
+  ps->counters[1] += w.nupd;
+  ps->counters[2] += w.ndst;
+  ps->counters[3] += 1;
+  w.used_slots.clear();
+  w.nupd = w.ndst = 0;
+  if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+  return 0;
 }
 
 int do_step(rudra_ps* ps, float* const* dsts, uint32_t k) {
@@ -171,23 +220,10 @@ int do_step(rudra_ps* ps, float* const* dsts, uint32_t k) {
   if (ps->queue.size() < ps->c) return 0;   // group still open: nothing changes
   DeviceScope dev(ps->device);
   if (!dev.ok()) return fail(RUDRA_E_CUDA, "cannot select device %d", ps->device);
-  rudra::UpdateParams p;
-  close_group(ps, p);
-  p.ndst = k;
-  for (uint32_t d = 0; d < k; ++d) p.dst[d] = dsts[d];
-  p.reverse = ps->sweep++ & 1u;
-  cudaError_t e = rudra::launch_update(p, ps->gtype == RUDRA_GRAD_BF16 ? rudra::kBF16 : rudra::kF32,
-                                       ps->optim == RUDRA_OPTIM_ADAGRAD ? rudra::kAdagrad : rudra::kMomentumSgd,
-                                       ps->stream);
-  if (e != cudaSuccess) return cuda_fail(e, "update kernel launch");
-  for (uint32_t l = 0; l < ps->c; ++l) {
-    if (ps->queue.front().slot >= 0) ps->free_slots.push_back(ps->queue.front().slot);
-    ps->queue.pop_front();
-  }
-  ps->ts += 1;   // exactly one increment per weight update
-  ps->counters[1] += 1;
-  ps->counters[2] += k;
-  ps->counters[3] += 1;
+  Window w;
+  append_update(ps, w);
+  for (uint32_t d = 0; d < k; ++d) w.p.dst[w.ndst++] = dsts[d];
+  if (int r = flush_window(ps, w)) return r;
   return 1;
 }
 
@@ -346,6 +382,87 @@ int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_
 int rudra_ps_step(rudra_ps* ps) { return do_step(ps, nullptr, 0); }
 
 int rudra_ps_step_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) { return do_step(ps, dsts_dev, k); }
+
+int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t count,
+                            const void* const* grads_dev, float* const* slots_dev, uint32_t max_window) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (count && !events) return fail(RUDRA_E_INVAL, "null event list");
+  const uint32_t cap = max_window == 0 || max_window > (uint32_t)rudra::kMaxWindow ? (uint32_t)rudra::kMaxWindow : max_window;
+  // Pass 1: replay the integers only.  Nothing is queued or launched unless the whole batch is legal.
+  {
+    uint64_t ts = ps->ts;
+    uint64_t queued = ps->queue.size();
+    for (uint64_t i = 0; i < count; ++i) {
+      const rudra_event& ev = events[i];
+      const bool needs_learner = ev.kind == RUDRA_EV_PUSH || ev.kind == RUDRA_EV_PULL;
+      if (needs_learner && ev.learner >= ps->lambda) return fail(RUDRA_E_INVAL, "event %llu: learner %u out of range", (unsigned long long)i, ev.learner);
+      switch (ev.kind) {
+        case RUDRA_EV_PUSH:
+          if (!grads_dev || !aligned(grads_dev[ev.learner])) return fail(RUDRA_E_INVAL, "event %llu: gradient buffer of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
+          if (ev.pulled_ts > ts) return fail(RUDRA_E_BAD_TS, "event %llu: pulled_ts %llu is ahead of the server timestamp %llu", (unsigned long long)i, (unsigned long long)ev.pulled_ts, (unsigned long long)ts);
+          if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: push expects server timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+          if (++queued > RUDRA_QUEUE_CAP) return fail(RUDRA_E_QUEUE_FULL, "event %llu: queue full", (unsigned long long)i);
+          break;
+        case RUDRA_EV_STEP:
+          if (queued < ps->c) return fail(RUDRA_E_STATE, "event %llu: update with %llu of %u gradients queued", (unsigned long long)i, (unsigned long long)queued, ps->c);
+          queued -= ps->c;
+          ts += 1;
+          if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: update expects new timestamp %llu, server reaches %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+          break;
+        case RUDRA_EV_PULL:
+          if (!slots_dev || !aligned(slots_dev[ev.learner])) return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
+          if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: pull expects timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+          break;
+        case RUDRA_EV_PULL_SKIP:
+          break;
+        case RUDRA_EV_BROADCAST:
+          if (!slots_dev) return fail(RUDRA_E_INVAL, "event %llu: broadcast without slots", (unsigned long long)i);
+          for (uint32_t l = 0; l < ps->lambda; ++l)
+            if (!aligned(slots_dev[l])) return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, l);
+          break;
+        default:
+          return fail(RUDRA_E_INVAL, "event %llu: unknown kind %d", (unsigned long long)i, ev.kind);
+      }
+    }
+  }
+  // Pass 2: handle the messages in order, packing consecutive updates and the pulls between them
+  // into one launch for as long as the launch tables have room.
+  DeviceScope dev(ps->device);
+  if (!dev.ok()) return fail(RUDRA_E_CUDA, "cannot select device %d", ps->device);
+  Window w;
+  int64_t updates = 0;
+  auto add_pull = [&](float* dst) -> int {
+    if (w.ndst == (uint32_t)rudra::kMaxDsts)
+      if (int r = flush_window(ps, w)) return r;
+    w.p.dst[w.ndst++] = dst;
+    return 0;
+  };
+  for (uint64_t i = 0; i < count; ++i) {
+    const rudra_event& ev = events[i];
+    switch (ev.kind) {
+      case RUDRA_EV_PUSH:
+        enqueue(ps, grads_dev[ev.learner], ev.pulled_ts, -1);
+        break;
+      case RUDRA_EV_STEP:
+        if (!window_has_room_for_update(ps, w, cap))
+          if (int r = flush_window(ps, w)) return r;
+        append_update(ps, w);
+        updates += 1;
+        break;
+      case RUDRA_EV_PULL:
+        if (int r = add_pull(slots_dev[ev.learner])) return r;
+        break;
+      case RUDRA_EV_BROADCAST:
+        for (uint32_t l = 0; l < ps->lambda; ++l)
+          if (int r = add_pull(slots_dev[l])) return r;
+        break;
+      default:
+        break;
+    }
+  }
+  if (int r = flush_window(ps, w)) return r;
+  return updates;
+}
 
 int64_t rudra_ps_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) {
   if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");

@@ -5,7 +5,9 @@
 // the c gradient values at index k.  So there is no reduction across threads, no shared memory
 // and no atomics; the kernel's only job is to keep enough bytes in flight to saturate HBM3e and
 // to touch every byte exactly once: c gradient reads, one read and one write of the weights and
-// of the state vector, and (optionally) ndst writes of the new weights into learner buffers.
+// of the state vector, and (optionally) writes of the new weights into learner buffers.  A launch
+// can carry a window of several consecutive updates: weights and state then stay in registers
+// from one update to the next, and the pulls between them become plain stores.
 //
 // A thread works on units of 8 consecutive weights.  fp32 vectors move with 256-bit global loads
 // and stores (ld/st.global.v8.f32, new with sm_100), bf16 gradients with 128-bit loads, so a
@@ -39,6 +41,14 @@ __device__ __forceinline__ F8 ld8(const float* p) {
 
 __device__ __forceinline__ void st8(float* p, const F8& r) {
   asm volatile("st.global.L2::evict_last.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
+               : "memory");
+}
+
+// Pull destinations are written once and not read again by the server: keep them out of the way
+// of the weights and state in L2.
+__device__ __forceinline__ void st8_stream(float* p, const F8& r) {
+  asm volatile("st.global.L2::evict_first.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
                :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
                : "memory");
 }
@@ -105,20 +115,25 @@ __device__ __forceinline__ void accumulate(const UpdateParams& p, uint32_t l0, u
 // AdaGrad: g = acc + wd theta (acc already the weighted mean gradient); h' = h + g^2;
 // theta' = theta - (sum s) g / (sqrt(h') + eps).
 template <int OPT, bool STATE>
-__device__ __forceinline__ void apply(const UpdateParams& p, float acc, float& theta, float& state) {
+__device__ __forceinline__ void apply(const UpdateParams& p, float awd, float abar, float acc, float& theta,
+                                      float& state) {
   if (OPT == kMomentumSgd) {
-    const float u = fmaf(p.awd, theta, acc);
+    const float u = fmaf(awd, theta, acc);
     const float v = STATE ? fmaf(p.momentum, state, u) : u;
     theta = theta - v;
     state = v;
   } else {
     const float g = fmaf(p.wd, theta, acc);
     const float h = fmaf(g, g, state);
-    theta = theta - __fdiv_rn(p.abar * g, __fsqrt_rn(h) + p.eps);
+    theta = theta - __fdiv_rn(abar * g, __fsqrt_rn(h) + p.eps);
     state = h;
   }
 }
 
+// A thread's units through the whole window: weights and state are loaded once, carried in
+// registers across the nupd updates and stored once; each update streams its own c gradients and
+// the pulls that follow it are stores of the registers.  Weights never interact, so this is the
+// same arithmetic, in the same order, as nupd separate launches.
 template <typename G, int OPT, bool STATE, int KMAX, int U, int THREADS, bool GUARD>
 __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t unit0, uint64_t nunits) {
   F8 th[U], st[U];
@@ -130,34 +145,57 @@ __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t uni
       th[j] = ld8(p.theta + u * kUnit);
       if (STATE) st[j] = ld8(p.state + u * kUnit);
     }
+  }
+  uint32_t d = 0;
+  for (const uint32_t d1 = p.dst_end[0]; d < d1; ++d) {   // pulls that arrived before the first update
 #pragma unroll
-    for (int e = 0; e < kUnit; ++e) acc[j][e] = 0.f;
+    for (int j = 0; j < U; ++j) {
+      const uint64_t u = unit0 + (uint64_t)j * THREADS;
+      if (!GUARD || u < nunits) st8_stream(p.dst[d] + u * kUnit, th[j]);
+    }
   }
   uint32_t l = 0;
-  for (; l + KMAX <= p.c; l += KMAX) accumulate<G, KMAX, U, THREADS, GUARD>(p, l, unit0, nunits, acc);
-  switch (p.c - l) {   // uniform across the grid
-    case 7: if (KMAX > 7) accumulate<G, 7, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-    case 6: if (KMAX > 6) accumulate<G, 6, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-    case 5: if (KMAX > 5) accumulate<G, 5, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-    case 4: if (KMAX > 4) accumulate<G, 4, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-    case 3: if (KMAX > 3) accumulate<G, 3, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-    case 2: if (KMAX > 2) accumulate<G, 2, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-    case 1: accumulate<G, 1, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-    default: break;
+  for (uint32_t w = 0; w < p.nupd; ++w) {
+#pragma unroll
+    for (int j = 0; j < U; ++j)
+#pragma unroll
+      for (int e = 0; e < kUnit; ++e) acc[j][e] = 0.f;
+    const uint32_t l1 = l + p.c;
+    for (; l + KMAX <= l1; l += KMAX) accumulate<G, KMAX, U, THREADS, GUARD>(p, l, unit0, nunits, acc);
+    switch (l1 - l) {   // uniform across the grid
+      case 7: if (KMAX > 7) accumulate<G, 7, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+      case 6: if (KMAX > 6) accumulate<G, 6, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+      case 5: if (KMAX > 5) accumulate<G, 5, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+      case 4: if (KMAX > 4) accumulate<G, 4, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+      case 3: if (KMAX > 3) accumulate<G, 3, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+      case 2: if (KMAX > 2) accumulate<G, 2, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+      case 1: accumulate<G, 1, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
+      default: break;
+    }
+    l = l1;
+    const float awd = p.awd[w], abar = p.abar[w];
+#pragma unroll
+    for (int j = 0; j < U; ++j)
+#pragma unroll
+      for (int e = 0; e < kUnit; ++e) {
+        float s = STATE ? st[j].v[e] : 0.f;
+        apply<OPT, STATE>(p, awd, abar, acc[j][e], th[j].v[e], s);
+        if (STATE) st[j].v[e] = s;
+      }
+    for (const uint32_t d1 = p.dst_end[w + 1]; d < d1; ++d) {   // pulls that follow this update
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+        const uint64_t u = unit0 + (uint64_t)j * THREADS;
+        if (!GUARD || u < nunits) st8_stream(p.dst[d] + u * kUnit, th[j]);
+      }
+    }
   }
 #pragma unroll
   for (int j = 0; j < U; ++j) {
     const uint64_t u = unit0 + (uint64_t)j * THREADS;
     if (!GUARD || u < nunits) {
-#pragma unroll
-      for (int e = 0; e < kUnit; ++e) {
-        float s = STATE ? st[j].v[e] : 0.f;
-        apply<OPT, STATE>(p, acc[j][e], th[j].v[e], s);
-        if (STATE) st[j].v[e] = s;
-      }
       st8(p.theta + u * kUnit, th[j]);
       if (STATE) st8(p.state + u * kUnit, st[j]);
-      for (uint32_t d = 0; d < p.ndst; ++d) st8(p.dst[d] + u * kUnit, th[j]);
     }
   }
 }
@@ -175,14 +213,18 @@ __global__ void __launch_bounds__(THREADS) update_kernel(const __grid_constant__
     process_tile<G, OPT, STATE, KMAX, U, THREADS, true>(p, tile * kTile + threadIdx.x, nunits);
   const uint64_t k = nunits * kUnit + threadIdx.x;
   if (tile == 0 && k < p.n) {
-    float acc = 0.f;
-    for (uint32_t l = 0; l < p.c; ++l) acc = fmaf(p.scale[l], GradUnit<G>::scalar(p.grad[l], k), acc);
     float th = p.theta[k];
     float s = STATE ? p.state[k] : 0.f;
-    apply<OPT, STATE>(p, acc, th, s);
+    uint32_t d = 0, l = 0;
+    for (const uint32_t d1 = p.dst_end[0]; d < d1; ++d) p.dst[d][k] = th;
+    for (uint32_t w = 0; w < p.nupd; ++w) {
+      float acc = 0.f;
+      for (const uint32_t l1 = l + p.c; l < l1; ++l) acc = fmaf(p.scale[l], GradUnit<G>::scalar(p.grad[l], k), acc);
+      apply<OPT, STATE>(p, p.awd[w], p.abar[w], acc, th, s);
+      for (const uint32_t d1 = p.dst_end[w + 1]; d < d1; ++d) p.dst[d][k] = th;
+    }
     p.theta[k] = th;
     if (STATE) p.state[k] = s;
-    for (uint32_t d = 0; d < p.ndst; ++d) p.dst[d][k] = th;
   }
 }
 
