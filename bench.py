@@ -34,6 +34,34 @@ UNIT = "updates/s"
 FALLBACK_HBM_GBS = 6650.0
 
 
+# DRAM traffic per weight of one launch of the dominant kernel, from ncu captures summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller vector; traffic grows in
+# proportion to the vector length).  Valid only for the kernel sources they were taken on.
+NCU_TRAFFIC = {
+    ("imagenet", 18): {"bytes_per_weight": 438.6, "kernel_sha": "67f846691f28f5ca",
+                       "source": "profiles/update_kernel_imagenet_window18.md"},
+}
+
+
+def kernel_sources_sha():
+    import hashlib
+
+    h = hashlib.sha256()
+    for f in ("update.cu", "kernels.cuh"):
+        with open(os.path.join(ROOT, "paper_1509_04210_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload, window, nparams):
+    """Bytes per launch from the recorded capture, or None if there is none for this shape or the
+    kernel has changed since."""
+    rec = NCU_TRAFFIC.get((workload, window))
+    if rec is None or rec["kernel_sha"] != kernel_sources_sha():
+        return None
+    return rec["bytes_per_weight"] * nparams
+
+
 def measured_hbm_peak():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -420,7 +448,7 @@ def run_ours(args, w):
                 "peak_kind": "of %s" % peak_kind, "launches_timed": len(timed), "avg_launch_us": upd_ms * 1e3,
                 "bytes_per_launch": kern_bytes / max(len(timed), 1),
                 "frac_of_8TBs_datasheet": achieved / 8000.0,
-                "traffic": None,
+                "traffic": ncu_traffic(w.name, W, N),
             },
         }
         if world == 1 and not args.no_cpu_baseline and not args.kernel_only:
