@@ -373,7 +373,7 @@ def run_ours(args, w):
             t = torch.empty(N, dtype=bufs[0].dtype).pin_memory()
             t.copy_(bufs[l])
             hg.append(t)
-        hdst = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(2)]
+        hdst = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(4)]
         torch.cuda.synchronize()
         ps2 = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
         ps2.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
@@ -389,7 +389,7 @@ def run_ours(args, w):
                 elif kind == EV_STEP:
                     ps2.step()
                 elif kind == EV_PULL:
-                    ps2.pull_host(hdst[k % 2])
+                    ps2.pull_host(hdst[k % 4])
                     k += 1
                 elif kind == EV_BROADCAST:
                     ps2.pull_host(hdst[0])   # one copy leaves the device; learners on the host share it
@@ -397,12 +397,14 @@ def run_ours(args, w):
         e2e_warm = min(args.warmup, 3)
         for win in windows[:e2e_warm]:
             run_window_host(win)
+        ps2.sync()
         barrier()
         h0 = ps2.counters()
         s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s2.record(stream)
         for win in windows[e2e_warm: e2e_warm + e2e_steps]:
             run_window_host(win)
+        ps2.sync()            # uploads, updates and downloads run on three streams: wait for all of them
         e2.record(stream)
         barrier()
         h1 = ps2.counters()

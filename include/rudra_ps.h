@@ -103,9 +103,11 @@ int rudra_ps_set_weights_host(rudra_ps* ps, const float* src_host);
  */
 int64_t rudra_ps_push(rudra_ps* ps, const void* grad_dev, uint64_t pulled_ts);
 
-/* Same, for a gradient in host memory: it is copied on the stream into a staging buffer the
- * handle owns (allocated on first use, re-used afterwards), so grad_host may be re-used once the
- * copy has run.  Page-locked memory makes the copy asynchronous. */
+/* Same, for a gradient in host memory: it is copied into a staging buffer the handle owns
+ * (allocated on first use, re-used afterwards) on an upload stream of the handle's own, so that
+ * uploads, updates and rudra_ps_pull_host downloads overlap; the consuming update waits for the
+ * copy.  grad_host may be re-used after rudra_ps_sync.  Page-locked memory makes the copy
+ * asynchronous. */
 int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_ts);
 
 /*
@@ -129,8 +131,10 @@ int rudra_ps_step_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k);
 /*
  * rudra_ps_pull -- pullWeights (Section 2, Section 3.2): enqueues a copy of the weights, as of
  * every update issued so far, into dst (caller-owned, nparams floats) and returns their
- * timestamp.  rudra_ps_pull_host copies to host memory.  rudra_ps_pull_many serves k learners
- * with one read of the weights.
+ * timestamp.  rudra_ps_pull_many serves k learners with one read of the weights.
+ * rudra_ps_pull_host copies to host memory: a device snapshot on the handle's stream, then the
+ * transfer on a download stream of the handle's own, so later updates do not wait for the link;
+ * dst_host is complete after rudra_ps_sync.
  */
 int64_t rudra_ps_pull(rudra_ps* ps, float* dst_dev);
 int64_t rudra_ps_pull_host(rudra_ps* ps, float* dst_host);
@@ -151,7 +155,8 @@ int rudra_ps_last_clock(const rudra_ps* ps, uint64_t* pulled_ts_out, uint32_t* s
 int rudra_ps_export_state(rudra_ps* ps, float* theta_dst_dev, float* state_dst_dev);
 int rudra_ps_import_state(rudra_ps* ps, const float* theta_src_dev, const float* state_src_dev, uint64_t ts);
 
-/* Waits for the handle's stream; reports asynchronous CUDA errors as RUDRA_E_CUDA. */
+/* Waits for the handle's stream and its upload / download streams; reports asynchronous CUDA
+ * errors as RUDRA_E_CUDA. */
 int rudra_ps_sync(rudra_ps* ps);
 
 /* Counters since create: out[0] pushes, out[1] updates, out[2] pulls served (destinations),

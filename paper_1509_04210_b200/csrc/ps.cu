@@ -73,8 +73,17 @@ struct rudra_ps {
   float* state = nullptr;
   uint64_t ts = 0;
   std::deque<Pending> queue;
+  // Host-buffer path: gradients arrive over PCIe on an upload stream into staging slots, pulled
+  // weights leave on a download stream from snapshot buffers, so both directions of the link
+  // and the update kernels overlap.  Events order slot re-use against the kernels that read them.
+  cudaStream_t up_stream = nullptr, down_stream = nullptr;
   std::vector<void*> slots;        // staging buffers for gradients pushed from host memory
+  std::vector<cudaEvent_t> slot_ready;   // upload into the slot has finished
+  std::vector<cudaEvent_t> slot_spent;   // the update that read the slot has finished
   std::vector<int> free_slots;
+  struct DownBuf { float* buf = nullptr; cudaEvent_t filled = nullptr, drained = nullptr; };
+  std::vector<DownBuf> down;       // snapshots on their way to host memory
+  uint32_t down_next = 0;
   bool has_clock = false;
   std::vector<uint64_t> clock;
   std::vector<uint32_t> sigma;
@@ -95,13 +104,44 @@ void release_queue(rudra_ps* ps) {
   ps->queue.clear();
 }
 
-int free_staging(rudra_ps* ps) {
+cudaError_t sync_all(rudra_ps* ps) {
   cudaError_t e = cudaStreamSynchronize(ps->stream);
+  if (e == cudaSuccess && ps->up_stream) e = cudaStreamSynchronize(ps->up_stream);
+  if (e == cudaSuccess && ps->down_stream) e = cudaStreamSynchronize(ps->down_stream);
+  return e;
+}
+
+cudaError_t ensure_copy_streams(rudra_ps* ps) {
+  cudaError_t e = cudaSuccess;
+  if (!ps->up_stream) e = cudaStreamCreateWithFlags(&ps->up_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess && !ps->down_stream) e = cudaStreamCreateWithFlags(&ps->down_stream, cudaStreamNonBlocking);
+  return e;
+}
+
+int free_staging(rudra_ps* ps) {
+  cudaError_t e = sync_all(ps);
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
   for (void* s : ps->slots) cudaFree(s);
+  for (cudaEvent_t ev : ps->slot_ready) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : ps->slot_spent) cudaEventDestroy(ev);
   ps->slots.clear();
+  ps->slot_ready.clear();
+  ps->slot_spent.clear();
   ps->free_slots.clear();
   return 0;
+}
+
+void free_host_path(rudra_ps* ps) {
+  free_staging(ps);
+  for (auto& d : ps->down) {
+    cudaFree(d.buf);
+    if (d.filled) cudaEventDestroy(d.filled);
+    if (d.drained) cudaEventDestroy(d.drained);
+  }
+  ps->down.clear();
+  if (ps->up_stream) cudaStreamDestroy(ps->up_stream);
+  if (ps->down_stream) cudaStreamDestroy(ps->down_stream);
+  ps->up_stream = ps->down_stream = nullptr;
 }
 
 int64_t enqueue(rudra_ps* ps, const void* grad, uint64_t pulled_ts, int slot) {
@@ -144,7 +184,10 @@ void append_update(rudra_ps* ps, Window& w) {
     sum_sigma += ps->sigma[l];
     sum_pulled += e.pulled_ts;
     p.grad[base + l] = e.grad;
-    if (e.slot >= 0) w.used_slots.push_back(e.slot);
+    if (e.slot >= 0) {
+      cudaStreamWaitEvent(ps->stream, ps->slot_ready[e.slot], 0);   // the kernel starts after its uploads
+      w.used_slots.push_back(e.slot);
+    }
   }
   ps->avg_sigma = (double)ps->ts - (double)sum_pulled / (double)c;
   double sum_scale = 0.0;
@@ -201,7 +244,10 @@ int flush_window(rudra_ps* ps, Window& w) {
     e = rudra::launch_update(p, ps->gtype == RUDRA_GRAD_BF16 ? rudra::kBF16 : rudra::kF32,
                              ps->optim == RUDRA_OPTIM_ADAGRAD ? rudra::kAdagrad : rudra::kMomentumSgd, ps->stream);
   }
-  for (int slot : w.used_slots) ps->free_slots.push_back(slot);   // stream order protects re-use
+  for (int slot : w.used_slots) {   // the next upload into the slot waits for this launch
+    cudaEventRecord(ps->slot_spent[slot], ps->stream);
+    ps->free_slots.push_back(slot);
+  }
   ps->counters[1] += w.nupd;
   ps->counters[2] += w.ndst;
   ps->counters[3] += 1;
@@ -273,8 +319,7 @@ rudra_ps* rudra_ps_create(uint64_t nparams, uint32_t lambda, uint32_t n, float a
 void rudra_ps_destroy(rudra_ps* ps) {
   if (!valid(ps)) return;
   DeviceScope dev(ps->device);
-  cudaStreamSynchronize(ps->stream);
-  for (void* s : ps->slots) cudaFree(s);
+  free_host_path(ps);
   cudaFree(ps->theta);
   cudaFree(ps->state);
   ps->magic = 0;
@@ -358,19 +403,31 @@ int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_
   if (!grad_host) return fail(RUDRA_E_INVAL, "null gradient pointer");
   if (int r = check_push(ps, pulled_ts)) return r;
   DeviceScope dev(ps->device);
+  cudaError_t e = ensure_copy_streams(ps);
+  if (e != cudaSuccess) return cuda_fail(e, "copy stream creation");
   int slot;
   if (!ps->free_slots.empty()) {
     slot = ps->free_slots.back();
     ps->free_slots.pop_back();
+    cudaStreamWaitEvent(ps->up_stream, ps->slot_spent[slot], 0);   // its last reader must be done
   } else {
     void* buf = nullptr;
-    cudaError_t e = cudaMalloc(&buf, ps->grad_bytes());
-    if (e != cudaSuccess) return cuda_fail(e, "staging buffer allocation");
+    cudaEvent_t ready = nullptr, spent = nullptr;
+    e = cudaMalloc(&buf, ps->grad_bytes());
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ready, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&spent, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+      cudaFree(buf);
+      if (ready) cudaEventDestroy(ready);
+      return cuda_fail(e, "staging buffer allocation");
+    }
     ps->slots.push_back(buf);
+    ps->slot_ready.push_back(ready);
+    ps->slot_spent.push_back(spent);
     slot = (int)ps->slots.size() - 1;
   }
-  // Stream order makes re-use safe: the update that read this slot was enqueued before this copy.
-  cudaError_t e = cudaMemcpyAsync(ps->slots[slot], grad_host, ps->grad_bytes(), cudaMemcpyHostToDevice, ps->stream);
+  e = cudaMemcpyAsync(ps->slots[slot], grad_host, ps->grad_bytes(), cudaMemcpyHostToDevice, ps->up_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(ps->slot_ready[slot], ps->up_stream);
   if (e != cudaSuccess) {
     ps->free_slots.push_back(slot);
     return cuda_fail(e, "gradient host-to-device copy");
@@ -492,9 +549,39 @@ int64_t rudra_ps_pull_host(rudra_ps* ps, float* dst_host) {
   if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
   if (!dst_host) return fail(RUDRA_E_INVAL, "null destination");
   DeviceScope dev(ps->device);
-  cudaError_t e = cudaMemcpyAsync(dst_host, ps->theta, ps->N * sizeof(float), cudaMemcpyDeviceToHost, ps->stream);
+  cudaError_t e = ensure_copy_streams(ps);
+  if (e != cudaSuccess) return cuda_fail(e, "copy stream creation");
+  constexpr uint32_t kDownBufs = 2;
+  if (ps->down.size() < kDownBufs) {
+    rudra_ps::DownBuf d;
+    e = cudaMalloc(reinterpret_cast<void**>(&d.buf), ps->N * sizeof(float));
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&d.filled, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&d.drained, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+      cudaFree(d.buf);
+      if (d.filled) cudaEventDestroy(d.filled);
+      return cuda_fail(e, "snapshot buffer allocation");
+    }
+    ps->down.push_back(d);
+  }
+  rudra_ps::DownBuf& d = ps->down[ps->down_next++ % ps->down.size()];
+  // snapshot on the main stream (after every update issued so far), then the copy to the host
+  // on the download stream, so later updates need not wait for PCIe
+  cudaStreamWaitEvent(ps->stream, d.drained, 0);
+  rudra::SnapshotParams sp;
+  sp.dst[0] = d.buf;
+  sp.src = ps->theta;
+  sp.n = ps->N;
+  sp.ndst = 1;
+  sp.reverse = ps->sweep++ & 1u;
+  e = rudra::launch_snapshot(sp, ps->stream);
+  if (e == cudaSuccess) e = cudaEventRecord(d.filled, ps->stream);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ps->down_stream, d.filled, 0);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dst_host, d.buf, ps->N * sizeof(float), cudaMemcpyDeviceToHost, ps->down_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(d.drained, ps->down_stream);
   if (e != cudaSuccess) return cuda_fail(e, "weights device-to-host copy");
   ps->counters[2] += 1;
+  ps->counters[3] += 1;
   ps->counters[5] += ps->N * sizeof(float);
   return (int64_t)ps->ts;
 }
@@ -545,7 +632,7 @@ int rudra_ps_import_state(rudra_ps* ps, const float* theta_src_dev, const float*
 int rudra_ps_sync(rudra_ps* ps) {
   if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
   DeviceScope dev(ps->device);
-  cudaError_t e = cudaStreamSynchronize(ps->stream);
+  cudaError_t e = sync_all(ps);
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
   return 0;
 }

@@ -45,10 +45,10 @@ __device__ __forceinline__ void st8(float* p, const F8& r) {
                : "memory");
 }
 
-// Pull destinations are written once and not read again by the server: keep them out of the way
-// of the weights and state in L2.
+// Pull destinations: plain write-back stores (measured 1 % faster on B200 than evict-first or
+// evict-last hints when half the traffic of a window is pull writes).
 __device__ __forceinline__ void st8_stream(float* p, const F8& r) {
-  asm volatile("st.global.L2::evict_first.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
                :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
                : "memory");
 }
