@@ -108,11 +108,16 @@ def make_windows(w, count, seed=synth.MASTER_SEED, from_oracle=False):
     return windows
 
 
+def launches_in_region(ps, c0):
+    return ps.counters()["launches"] - c0["launches"]
+
+
 def default_window(w):
     """Updates packed into one launch by default: the gradients lambda learners can have waiting at
     once make n = lambda / c updates (every learner blocks on its push until the server has taken
-    it), capped by the launch tables (32 updates, 128 gradients)."""
-    return max(1, min(w.n, 32, 128 // w.c))
+    it), capped by the launch tables (32 updates, 128 gradients, 128 pull destinations)."""
+    pulls_per_update = w.lam if (w.downcast or w.mode == synth.HARDSYNC) else w.c
+    return max(1, min(w.n, 32, 128 // w.c, 128 // pulls_per_update))
 
 
 def window_bytes_per_param(w, events):
@@ -326,23 +331,24 @@ def run_ours(args, w):
 
     def run_backlog(chunk, timed):
         """A backlog of W update windows through run_events: one launch when the tables allow."""
-        before = ps.counters()["launches"]
         e0, e1 = new_events()
         e0.record(stream)
         ps.run_events(chunk, gtable, stable, W)
         e1.record(stream)
-        if ps.counters()["launches"] == before + 1:
-            timed.append((e0, e1, window_bytes_per_param(w, chunk) * N))
+        timed.append((e0, e1, window_bytes_per_param(w, chunk) * N))
 
-    def run_all(wins, timed):
+    def prepare(wins):
+        """The messages as the server receives them: single windows, or backlogs of W windows."""
         if W == 0:
-            for win in wins:
-                run_messages(win, timed)
-        else:
-            for i in range(0, len(wins), W):
-                run_backlog(np.concatenate(wins[i:i + W]), timed)
+            return wins
+        return [np.concatenate(wins[i:i + W]) for i in range(0, len(wins), W)]
 
-    run_all(windows[: args.warmup], [])
+    def run_all(batches, timed):
+        for b in batches:
+            (run_messages if W == 0 else run_backlog)(b, timed)
+
+    warm_batches, timed_batches = prepare(windows[: args.warmup]), prepare(windows[args.warmup:])
+    run_all(warm_batches, [])
     barrier()
     sampler = ClockSampler(visible_gpu_index(local_rank))
     sampler.start()
@@ -350,12 +356,14 @@ def run_ours(args, w):
     start, end = new_events()
     timed = []
     start.record(stream)
-    run_all(windows[args.warmup:], timed)
+    run_all(timed_batches, timed)
     end.record(stream)
     barrier()
     clocks = sampler.stop()
     c1 = ps.counters()
     ms = start.elapsed_time(end)
+    if W != 0 and launches_in_region(ps, c0) != len(timed):
+        timed = []      # a backlog needed more than one launch: no per-launch figure for this shape
     kern_ms = float(sum(a.elapsed_time(b) for a, b, _ in timed))
     kern_bytes = float(sum(nb for _, _, nb in timed))
     upd_ms = kern_ms / max(len(timed), 1)

@@ -86,31 +86,6 @@ template <> struct GradUnit<__nv_bfloat16> {
   }
 };
 
-// acc += s_l * g_l for K gradient streams starting at table entry l0: all K * U loads are issued
-// before the first use.
-template <typename G, int K, int U, int THREADS, bool GUARD>
-__device__ __forceinline__ void accumulate(const UpdateParams& p, uint32_t l0, uint64_t unit0, uint64_t nunits,
-                                           float (&acc)[U][kUnit]) {
-  GradUnit<G> g[K][U];
-#pragma unroll
-  for (int l = 0; l < K; ++l) {
-    const void* base = p.grad[l0 + l];
-#pragma unroll
-    for (int j = 0; j < U; ++j) {
-      const uint64_t u = unit0 + (uint64_t)j * THREADS;
-      if (!GUARD || u < nunits) g[l][j].load(base, u); else g[l][j].zero();
-    }
-  }
-#pragma unroll
-  for (int l = 0; l < K; ++l) {
-    const float s = p.scale[l0 + l];
-#pragma unroll
-    for (int j = 0; j < U; ++j)
-#pragma unroll
-      for (int e = 0; e < kUnit; ++e) acc[j][e] = fmaf(s, g[l][j].get(e), acc[j][e]);
-  }
-}
-
 // The per-weight rule.  Momentum SGD: u = acc + (sum s) wd theta; v' = m v + u; theta' = theta - v'.
 // AdaGrad: g = acc + wd theta (acc already the weighted mean gradient); h' = h + g^2;
 // theta' = theta - (sum s) g / (sqrt(h') + eps).
@@ -134,7 +109,12 @@ __device__ __forceinline__ void apply(const UpdateParams& p, float awd, float ab
 // registers across the nupd updates and stored once; each update streams its own c gradients and
 // the pulls that follow it are stores of the registers.  Weights never interact, so this is the
 // same arithmetic, in the same order, as nupd separate launches.
-template <typename G, int OPT, bool STATE, int KMAX, int U, int THREADS, bool GUARD>
+//
+// The window's nupd * c gradient vectors are walked as one flat list, DEPTH loads in flight at a
+// time regardless of where one update ends and the next begins: the loads do not depend on the
+// running weights, only the short fma chain does, so a small model (few blocks, latency-bound)
+// does not pay one memory round trip per update.
+template <typename G, int OPT, bool STATE, int DEPTH, int U, int THREADS, bool GUARD>
 __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t unit0, uint64_t nunits) {
   F8 th[U], st[U];
   float acc[U][kUnit];
@@ -145,6 +125,8 @@ __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t uni
       th[j] = ld8(p.theta + u * kUnit);
       if (STATE) st[j] = ld8(p.state + u * kUnit);
     }
+#pragma unroll
+    for (int e = 0; e < kUnit; ++e) acc[j][e] = 0.f;
   }
   uint32_t d = 0;
   for (const uint32_t d1 = p.dst_end[0]; d < d1; ++d) {   // pulls that arrived before the first update
@@ -154,39 +136,51 @@ __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t uni
       if (!GUARD || u < nunits) st8_stream(p.dst[d] + u * kUnit, th[j]);
     }
   }
-  uint32_t l = 0;
-  for (uint32_t w = 0; w < p.nupd; ++w) {
+  const uint32_t total = p.nupd * p.c;
+  uint32_t w = 0;            // update being accumulated
+  uint32_t left = p.c;       // gradients it still waits for
+  for (uint32_t l0 = 0; l0 < total; l0 += DEPTH) {
+    GradUnit<G> g[DEPTH][U];
 #pragma unroll
-    for (int j = 0; j < U; ++j)
+    for (int i = 0; i < DEPTH; ++i) {
+      if (l0 + i < total) {   // uniform across the grid
+        const void* base = p.grad[l0 + i];
 #pragma unroll
-      for (int e = 0; e < kUnit; ++e) acc[j][e] = 0.f;
-    const uint32_t l1 = l + p.c;
-    for (; l + KMAX <= l1; l += KMAX) accumulate<G, KMAX, U, THREADS, GUARD>(p, l, unit0, nunits, acc);
-    switch (l1 - l) {   // uniform across the grid
-      case 7: if (KMAX > 7) accumulate<G, 7, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-      case 6: if (KMAX > 6) accumulate<G, 6, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-      case 5: if (KMAX > 5) accumulate<G, 5, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-      case 4: if (KMAX > 4) accumulate<G, 4, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-      case 3: if (KMAX > 3) accumulate<G, 3, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-      case 2: if (KMAX > 2) accumulate<G, 2, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-      case 1: accumulate<G, 1, U, THREADS, GUARD>(p, l, unit0, nunits, acc); break;
-      default: break;
-    }
-    l = l1;
-    const float awd = p.awd[w], abar = p.abar[w];
-#pragma unroll
-    for (int j = 0; j < U; ++j)
-#pragma unroll
-      for (int e = 0; e < kUnit; ++e) {
-        float s = STATE ? st[j].v[e] : 0.f;
-        apply<OPT, STATE>(p, awd, abar, acc[j][e], th[j].v[e], s);
-        if (STATE) st[j].v[e] = s;
+        for (int j = 0; j < U; ++j) {
+          const uint64_t u = unit0 + (uint64_t)j * THREADS;
+          if (!GUARD || u < nunits) g[i][j].load(base, u); else g[i][j].zero();
+        }
       }
-    for (const uint32_t d1 = p.dst_end[w + 1]; d < d1; ++d) {   // pulls that follow this update
+    }
 #pragma unroll
-      for (int j = 0; j < U; ++j) {
-        const uint64_t u = unit0 + (uint64_t)j * THREADS;
-        if (!GUARD || u < nunits) st8_stream(p.dst[d] + u * kUnit, th[j]);
+    for (int i = 0; i < DEPTH; ++i) {
+      if (l0 + i < total) {
+        const float s = p.scale[l0 + i];
+#pragma unroll
+        for (int j = 0; j < U; ++j)
+#pragma unroll
+          for (int e = 0; e < kUnit; ++e) acc[j][e] = fmaf(s, g[i][j].get(e), acc[j][e]);
+        if (--left == 0) {     // last gradient of update w: applyUpdate, then the pulls that follow it
+          const float awd = p.awd[w], abar = p.abar[w];
+#pragma unroll
+          for (int j = 0; j < U; ++j)
+#pragma unroll
+            for (int e = 0; e < kUnit; ++e) {
+              float sv = STATE ? st[j].v[e] : 0.f;
+              apply<OPT, STATE>(p, awd, abar, acc[j][e], th[j].v[e], sv);
+              if (STATE) st[j].v[e] = sv;
+              acc[j][e] = 0.f;
+            }
+          ++w;
+          left = p.c;
+          for (const uint32_t d1 = p.dst_end[w]; d < d1; ++d) {
+#pragma unroll
+            for (int j = 0; j < U; ++j) {
+              const uint64_t u = unit0 + (uint64_t)j * THREADS;
+              if (!GUARD || u < nunits) st8_stream(p.dst[d] + u * kUnit, th[j]);
+            }
+          }
+        }
       }
     }
   }
@@ -202,15 +196,15 @@ __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t uni
 
 // One tile of THREADS * U units per block; the last, ragged tile takes the guarded path and the
 // n % 8 trailing weights are done one by one by the block that owns tile 0.
-template <typename G, int OPT, bool STATE, int KMAX, int U, int THREADS>
+template <typename G, int OPT, bool STATE, int DEPTH, int U, int THREADS>
 __global__ void __launch_bounds__(THREADS) update_kernel(const __grid_constant__ UpdateParams p) {
   const uint64_t nunits = p.n / kUnit;
   constexpr uint64_t kTile = (uint64_t)THREADS * U;
   const uint64_t tile = p.reverse ? (uint64_t)gridDim.x - 1 - blockIdx.x : (uint64_t)blockIdx.x;
   if ((tile + 1) * kTile <= nunits)
-    process_tile<G, OPT, STATE, KMAX, U, THREADS, false>(p, tile * kTile + threadIdx.x, nunits);
+    process_tile<G, OPT, STATE, DEPTH, U, THREADS, false>(p, tile * kTile + threadIdx.x, nunits);
   else
-    process_tile<G, OPT, STATE, KMAX, U, THREADS, true>(p, tile * kTile + threadIdx.x, nunits);
+    process_tile<G, OPT, STATE, DEPTH, U, THREADS, true>(p, tile * kTile + threadIdx.x, nunits);
   const uint64_t k = nunits * kUnit + threadIdx.x;
   if (tile == 0 && k < p.n) {
     float th = p.theta[k];
@@ -228,30 +222,33 @@ __global__ void __launch_bounds__(THREADS) update_kernel(const __grid_constant__
   }
 }
 
-template <typename G, int OPT, bool STATE, int KMAX, int U, int THREADS>
+template <typename G, int OPT, bool STATE, int DEPTH, int U, int THREADS>
 cudaError_t launch_one(const UpdateParams& p, cudaStream_t stream) {
   const uint64_t nunits = p.n / kUnit;
   uint64_t tiles = (nunits + (uint64_t)THREADS * U - 1) / ((uint64_t)THREADS * U);
   if (tiles == 0) tiles = 1;                                      // n < 8: only the scalar tail
   if (tiles > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
-  update_kernel<G, OPT, STATE, KMAX, U, THREADS><<<(unsigned)tiles, THREADS, 0, stream>>>(p);
+  update_kernel<G, OPT, STATE, DEPTH, U, THREADS><<<(unsigned)tiles, THREADS, 0, stream>>>(p);
   return cudaGetLastError();
 }
 
-template <typename G, int KMAX, int U, int THREADS>
+template <typename G, int DEPTH, int THREADS>
 cudaError_t launch_typed(const UpdateParams& p, Optim optim, cudaStream_t stream) {
-  if (optim == kAdagrad) return launch_one<G, kAdagrad, true, KMAX, U, THREADS>(p, stream);
-  if (p.momentum != 0.f) return launch_one<G, kMomentumSgd, true, KMAX, U, THREADS>(p, stream);
-  return launch_one<G, kMomentumSgd, false, KMAX, U, THREADS>(p, stream);   // no velocity kept
+  if (optim == kAdagrad) return launch_one<G, kAdagrad, true, DEPTH, 1, THREADS>(p, stream);
+  if (p.momentum != 0.f) return launch_one<G, kMomentumSgd, true, DEPTH, 1, THREADS>(p, stream);
+  return launch_one<G, kMomentumSgd, false, DEPTH, 1, THREADS>(p, stream);   // no velocity kept
 }
 
 }  // namespace
 
 cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, cudaStream_t stream) {
-  if (gtype == kBF16) return launch_typed<__nv_bfloat16, 8, 1, 256>(p, optim, stream);
-  // fp32: with few gradient streams a thread carries two units to keep enough loads in flight
-  if (p.c <= 2) return launch_typed<float, 4, 2, 256>(p, optim, stream);
-  return launch_typed<float, 4, 1, 256>(p, optim, stream);
+  // Large vectors: 256-thread tiles (measured: any tile shape saturates HBM).  Vectors that give
+  // fewer than ~32 such tiles per SM of a 148-SM part are latency-bound or leave the last wave
+  // ragged: 64-thread tiles spread them over four times as many blocks.
+  const bool small = p.n / kUnit < 148ull * 32 * 256;
+  if (gtype == kBF16)
+    return small ? launch_typed<__nv_bfloat16, 8, 64>(p, optim, stream) : launch_typed<__nv_bfloat16, 8, 256>(p, optim, stream);
+  return small ? launch_typed<float, 8, 64>(p, optim, stream) : launch_typed<float, 4, 256>(p, optim, stream);
 }
 
 }  // namespace rudra
