@@ -22,6 +22,11 @@
 //                                           : parity unpinned by the paper.
 // Everything else is pinned by Eq. 2-6 and the staleness sets printed in
 // Section 5.1 (see tests/).
+//
+// A second evaluation mode ("strict") carries the same rule in fp32 with one
+// fused multiply-add per term, gradients in arrival order.  It is a debugging
+// aid that lets an fp32 implementation be compared bit for bit; the parity
+// criterion is the double-precision mode.
 #include <algorithm>
 #include <cmath>
 #include <cstdint>
@@ -205,6 +210,7 @@ struct OraclePS {
   int32_t dtype = GRAD_F32;
   int32_t optimizer = OPT_MOMENTUM_SGD;
   float adagrad_eps = 1e-8f;
+  bool strict = false;             // fp32 evaluation, one fmaf per term (debugging aid)
   std::vector<float> theta, vel;   // vel: velocity (momentum SGD) or squared-gradient sum (AdaGrad)
   uint64_t ts = 0;
   std::deque<Pending> fifo;
@@ -265,6 +271,12 @@ struct OraclePS {
     }
     abar = (float)sum_s;   // the group's learning rate: sum of the per-gradient step sizes
 
+    if (strict) {
+      step_strict(grp);
+      ts += 1;
+      fifo.erase(fifo.begin(), fifo.begin() + c);
+      return 1;
+    }
     for (uint64_t k = 0; k < N; ++k) {
       if (optimizer == OPT_MOMENTUM_SGD) {
         // sumGradients: staleness-scaled average of the c gradients (Eq. 5 with Eq. 6 folded in)
@@ -293,6 +305,33 @@ struct OraclePS {
     ts += 1;   // each weight update increments the timestamp by one (Section 3.1)
     fifo.erase(fifo.begin(), fifo.begin() + c);
     return 1;
+  }
+
+  // The same rule in fp32: acc = fma(s_l, g_l, acc) for l = 1..c from acc = 0, then one fma per
+  // remaining term.  Same reading of momentum / decay / AdaGrad as above.
+  void step_strict(const std::vector<Pending>& grp) {
+    const float awd = (float)((double)abar * (double)wd);
+    for (uint64_t k = 0; k < N; ++k) {
+      float acc = 0.f;
+      if (optimizer == OPT_MOMENTUM_SGD) {
+        for (uint32_t l = 0; l < c; ++l) acc = std::fmaf(scale[l], (float)grad_at(grp[l].grad, k), acc);
+        const float u = std::fmaf(awd, theta[k], acc);
+        const float v = momentum != 0.f ? std::fmaf(momentum, vel[k], u) : u;
+        theta[k] = theta[k] - v;
+        vel[k] = v;
+      } else {
+        for (uint32_t l = 0; l < c; ++l) {
+          const float wl = (float)((double)scale[l] / (double)abar);
+          acc = std::fmaf(wl, (float)grad_at(grp[l].grad, k), acc);
+        }
+        const float g = std::fmaf(wd, theta[k], acc);
+        const float h = std::fmaf(g, g, vel[k]);
+        const float num = abar * g;
+        const float den = std::sqrt(h) + adagrad_eps;
+        theta[k] = theta[k] - num / den;
+        vel[k] = h;
+      }
+    }
   }
 
   int64_t pull(float* dst) const {   // pullWeights: the weights and their timestamp (Section 3.2)
@@ -335,6 +374,7 @@ void ora_ps_set_optimizer(void* p, int32_t opt, float eps) {
   ((OraclePS*)p)->optimizer = opt;
   ((OraclePS*)p)->adagrad_eps = eps;
 }
+void ora_ps_set_strict(void* p, int32_t on) { ((OraclePS*)p)->strict = on != 0; }
 void ora_ps_set_alpha0(void* p, float a0) { ((OraclePS*)p)->alpha0 = a0; }
 void ora_ps_set_weights(void* p, const float* src) {
   OraclePS* P = (OraclePS*)p;

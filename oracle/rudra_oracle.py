@@ -57,6 +57,7 @@ def lib():
         L.ora_ps_set_grad_dtype.argtypes = [C.c_void_p, C.c_int32]
         L.ora_ps_set_optimizer.argtypes = [C.c_void_p, C.c_int32, C.c_float]
         L.ora_ps_set_alpha0.argtypes = [C.c_void_p, C.c_float]
+        L.ora_ps_set_strict.argtypes = [C.c_void_p, C.c_int32]
         L.ora_ps_set_weights.argtypes = [C.c_void_p, C.c_void_p]
         L.ora_ps_push.restype = C.c_int64
         L.ora_ps_push.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
@@ -121,6 +122,10 @@ class OraclePS:
 
     def set_alpha0(self, a0):
         lib().ora_ps_set_alpha0(self._h, a0)
+
+    def set_strict(self, on=True):
+        """fp32 evaluation with one fused multiply-add per term (debugging aid, not the parity bar)."""
+        lib().ora_ps_set_strict(self._h, int(bool(on)))
 
     def set_weights(self, theta0):
         a = np.ascontiguousarray(theta0, dtype=np.float32)

@@ -88,6 +88,27 @@ def test_adagrad_parity():
     pair.close()
 
 
+@pytest.mark.parametrize("dtype,optimizer", [(synth.GRAD_F32, ora.OPT_MOMENTUM_SGD), (synth.GRAD_BF16, ora.OPT_MOMENTUM_SGD),
+                                             (synth.GRAD_F32, ora.OPT_ADAGRAD)])
+def test_bit_exact_against_the_fp32_evaluation_of_the_oracle(dtype, optimizer):
+    # Not the parity bar (that is the double-precision oracle, above) but a sharper net: the kernel
+    # has no cross-thread reduction, so with the oracle evaluating the same rule in fp32, one fma
+    # per term in arrival order, every weight and state value must agree to the last bit.
+    N, lam, n = 70003, 15, 3
+    pair = Pair(N, lam, n, 0.03, 0.9 if optimizer == ora.OPT_MOMENTUM_SGD else 0.0, 5e-4, dtype,
+                policy=ora.LR_PER_GRADIENT, optimizer=optimizer)
+    pair.cpu.set_strict(True)
+    rng = np.random.default_rng(8)
+    for step in range(6):
+        for l in range(5):
+            pair.push(synth.gradient(N, l, step, 1e-2, dtype), int(rng.integers(0, pair.gpu.timestamp() + 1)))
+        assert pair.step() == 1
+        th, st = pair.weights()
+        np.testing.assert_array_equal(th.view(np.uint32), pair.cpu.pull()[0].view(np.uint32))
+        np.testing.assert_array_equal(st.view(np.uint32), pair.cpu.state().view(np.uint32))
+    pair.close()
+
+
 def test_pull_variants_are_exact_copies():
     import torch
 

@@ -305,3 +305,26 @@ def test_adagrad_constant_gradient_closed_form():
     want = th0 - a * sum(g64 / (np.sqrt(j) * np.abs(g64) + eps) for j in range(1, K + 1))
     _close(ps.pull()[0], want, 1e-2, ulps=2.0 * K)
     _close(ps.state(), K * g64 * g64, 0.0, ulps=2.0 * K)
+
+
+def test_strict_fp32_mode_tracks_the_double_mode():
+    # the fp32 evaluation is the same rule: after a few updates it differs only by fp32 rounding
+    N, lam, n = 500, 6, 2
+    for opt in (ora.OPT_MOMENTUM_SGD, ora.OPT_ADAGRAD):
+        a, _ = _mk(N, lam, n, 0.02, m=0.9 if opt == ora.OPT_MOMENTUM_SGD else 0.0, wd=5e-4)
+        b, _ = _mk(N, lam, n, 0.02, m=0.9 if opt == ora.OPT_MOMENTUM_SGD else 0.0, wd=5e-4)
+        for ps in (a, b):
+            ps.set_optimizer(opt, 1e-8)
+            ps.set_policy(ora.LR_PER_GRADIENT)
+        b.set_strict(True)
+        for k in range(10):
+            for l in range(3):
+                g = synth.gradient(N, l, k, 1e-2)
+                p_ts = max(0, a.timestamp() - l)
+                a.push(g, p_ts)
+                b.push(g, p_ts)
+            assert a.step() == 1 and b.step() == 1
+        ta, tb = a.pull()[0].astype(np.float64), b.pull()[0].astype(np.float64)
+        rms = np.sqrt(np.mean(ta * ta))
+        assert np.max(np.abs(ta - tb) / np.maximum(np.abs(ta), rms)) < 2e-6
+        assert not np.array_equal(a.pull()[0], b.pull()[0]) or opt == ora.OPT_ADAGRAD
