@@ -243,9 +243,9 @@ cudaError_t launch_typed(const UpdateParams& p, Optim optim, cudaStream_t stream
 
 cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, cudaStream_t stream) {
   // Large vectors: 256-thread tiles (measured: any tile shape saturates HBM).  Vectors that give
-  // fewer than ~32 such tiles per SM of a 148-SM part are latency-bound or leave the last wave
+  // fewer than ~16 such tiles per SM of a 148-SM part are latency-bound or leave the last wave
   // ragged: 64-thread tiles spread them over four times as many blocks.
-  const bool small = p.n / kUnit < 148ull * 32 * 256;
+  const bool small = p.n / kUnit < 148ull * 16 * 256;
   if (gtype == kBF16)
     return small ? launch_typed<__nv_bfloat16, 8, 64>(p, optim, stream) : launch_typed<__nv_bfloat16, 8, 256>(p, optim, stream);
   return small ? launch_typed<float, 8, 64>(p, optim, stream) : launch_typed<float, 4, 256>(p, optim, stream);
