@@ -70,11 +70,19 @@ def measured_hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+ADAGRAD = False   # set from --optimizer
+
+
+def state_bytes(w):
+    """Read + write of the weights, and of the state vector when the rule keeps one (velocity with
+    momentum, squared-gradient sum with AdaGrad)."""
+    return 16 if (w.momentum != 0.0 or ADAGRAD) else 8
+
+
 def update_bytes_per_param(w):
-    """Algorithmic bytes one update moves per weight: c gradient reads + read and write of the
-    weights and (with momentum) of the velocity."""
+    """Algorithmic bytes one update moves per weight: c gradient reads + weights and state."""
     g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
-    return w.c * g + (16 if w.momentum != 0.0 else 8)
+    return w.c * g + state_bytes(w)
 
 
 EV_PUSH, EV_STEP, EV_PULL, EV_PULL_SKIP, EV_BROADCAST = 1, 2, 3, 4, 5
@@ -126,7 +134,7 @@ def window_bytes_per_param(w, events):
     g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
     pushes = int((events["kind"] == EV_STEP).sum()) * w.c
     pulls = int((events["kind"] == EV_PULL).sum()) + w.lam * int((events["kind"] == EV_BROADCAST).sum())
-    return pushes * g + (16 if w.momentum != 0.0 else 8) + 4 * pulls
+    return pushes * g + state_bytes(w) + 4 * pulls
 
 
 class ClockSampler(threading.Thread):
@@ -195,13 +203,15 @@ def visible_gpu_index(local_rank):
 # ---------------------------------------------------------------------------------------------
 # CPU oracle legs (the reported baseline and the --impl reference arm)
 # ---------------------------------------------------------------------------------------------
-def oracle_run(w, windows, nsample, grads_host, warmup=0, budget_s=None, max_windows=None):
+def oracle_run(w, windows, nsample, grads_host, warmup=0, budget_s=None, max_windows=None, adagrad=False):
     """Times the oracle, as it stands, over event windows (from the start of the event stream) on
     the first nsample weights; the first ``warmup`` windows run untimed."""
     from oracle import rudra_oracle as ora
 
     ps = ora.OraclePS(nsample, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
     ps.set_grad_dtype(w.grad_dtype)
+    if adagrad:
+        ps.set_optimizer(ora.OPT_ADAGRAD, 1e-8)
     ps.set_weights(synth.initial_weights(nsample, w.theta_std))
     done, t0 = -warmup, time.perf_counter()
     for win in windows:
@@ -240,7 +250,7 @@ def run_reference(args, w):
     nsample = max(1, w.nparams // 4) if w.nparams > (1 << 22) else w.nparams
     windows = make_windows(w, args.warmup + args.steps, from_oracle=True)
     grads = host_gradients(w, nsample, min(w.lam, 8))
-    done, dt = oracle_run(w, windows, nsample, grads, warmup=args.warmup)
+    done, dt = oracle_run(w, windows, nsample, grads, warmup=args.warmup, adagrad=args.optimizer == "adagrad")
     frac = nsample / w.nparams
     value = done / dt * frac
     sample = "first %d of %d weights (%.0f%%), %d distinct host gradient buffers, rate scaled by the fraction" % (
@@ -302,6 +312,8 @@ def run_ours(args, w):
     slots = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(nslots)]
     ps = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
     ps.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
+    if args.optimizer == "adagrad":
+        ps.set_option(rb.OPT_OPTIMIZER, rb.OPTIM_ADAGRAD)
     ps.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
     ps.sync()
     ps.set_stream(stream)
@@ -385,6 +397,8 @@ def run_ours(args, w):
         torch.cuda.synchronize()
         ps2 = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
         ps2.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
+        if args.optimizer == "adagrad":
+            ps2.set_option(rb.OPT_OPTIMIZER, rb.OPTIM_ADAGRAD)
         ps2.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
         ps2.sync()
         ps2.set_stream(stream)
@@ -426,11 +440,11 @@ def run_ours(args, w):
         g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
         achieved = kern_bytes / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else float("nan")
         # bytes the whole path must move per step: every gradient once, weights/state per launch, pulls
-        state_bytes = 16 if w.momentum != 0.0 else 8
+        sb = state_bytes(w)
         if W == 0:
-            path_bytes = N * (args.steps * (w.c * g + state_bytes) + 8 * pulls)
+            path_bytes = N * (args.steps * (w.c * g + sb) + 8 * pulls)
         else:
-            path_bytes = N * (args.steps * w.c * g + launches * state_bytes + 4 * pulls)
+            path_bytes = N * (args.steps * w.c * g + launches * sb + 4 * pulls)
         value = replicas.whole_job_rate(args.steps, world, ms)
         cfg = workload_config(w)
         cfg["window"] = W
@@ -468,7 +482,8 @@ def run_ours(args, w):
             nh = min(w.lam, 6)
             grads = [t.cpu().numpy() if w.grad_dtype == synth.GRAD_F32 else t.view(torch.int16).cpu().numpy().view(np.uint16)
                      for t in bufs[:nh]]
-            done, dt = oracle_run(w, windows, N, grads, warmup=1, budget_s=12.0, max_windows=args.steps)
+            done, dt = oracle_run(w, windows, N, grads, warmup=1, budget_s=12.0, max_windows=args.steps,
+                                  adagrad=args.optimizer == "adagrad")
             line["cpu_baseline"] = {
                 "value": done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
                 "sample": "%d full-size update windows of the same event stream (%d distinct gradient buffers), %.1f s"
@@ -484,13 +499,16 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=1800,
+                    help="timed update windows (default: 100 rounds of the 54 learners at the ImageNet-scale workload)")
+    ap.add_argument("--warmup", type=int, default=36)
     ap.add_argument("--workload", default="imagenet", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--window", type=int, default=-1,
                     help="update windows handed to the server per call: 0 = one message at a time, "
                          "-1 = what lambda blocked learners can have waiting (n = lambda/c updates)")
+    ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adagrad"],
+                    help="momentum SGD with weight decay (Section 4.2) or AdaGrad at the server (Section 5.5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-only", action="store_true",
                     help="device-resident timed region only: no end-to-end leg, no CPU baseline (profiler captures)")
@@ -501,6 +519,12 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     w = synth.WORKLOADS[args.workload]
+    if args.optimizer == "adagrad":
+        import dataclasses
+
+        global ADAGRAD
+        ADAGRAD = True
+        w = dataclasses.replace(w, name=w.name + "+adagrad", momentum=0.0)
     if args.nparams:
         import dataclasses
 

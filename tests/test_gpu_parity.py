@@ -316,3 +316,61 @@ def test_imagenet_config_full_size_sampled_fused_pulls():
 def test_stress_config_full_size_sampled():
     # 60 965 224 weights, bf16 gradients, lambda = 128, n = 4 (c = 32)
     _sampled_full_size(synth.WORKLOADS["stress"], 3, 20000, fused=True)
+
+
+def test_floor_group_size_lambda_30_n_4():
+    # the paper's own n = 4, lambda = 30 run (Section 5.1): c = floor(30 / 4) = 7
+    w = synth.Workload("l30n4", 12345, 30, 4, 0.01, 0.9, 5e-4, synth.SOFTSYNC_ROUNDS, 20, 0.01, 1e-2)
+    assert w.c == 7
+    run_workload(w, 20, check_every=5)
+    run_workload(w, 20, check_every=5, policy=ora.LR_GROUP_MEAN)
+
+
+def test_single_learner_is_plain_sgd_with_zero_staleness():
+    # lambda = 1: n-softsync degenerates to hardsync (Section 5.2); every sigma is 0
+    w = synth.Workload("l1", 3001, 1, 1, 0.05, 0.0, 0.0, synth.SOFTSYNC_ROUNDS, 10, 0.01, 1e-2)
+    errs = run_workload(w, 10, check_every=1, policy=ora.LR_PER_GRADIENT)
+    assert len(errs) == 10
+
+
+def test_two_handles_on_their_own_streams_do_not_interfere():
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    N = 200003
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    a = Pair(N, 4, 2, 0.05, 0.9, 5e-4, seed=1)
+    b = Pair(N, 6, 2, 0.02, 0.0, 1e-3, dtype=synth.GRAD_BF16, seed=2)
+    torch.cuda.synchronize()
+    a.gpu.set_stream(s1)
+    b.gpu.set_stream(s2)
+    for step in range(5):
+        for l in range(3):                       # interleave the two servers' messages
+            if l < 2:
+                a.push(synth.gradient(N, l, step, 1e-2, seed=1), a.gpu.timestamp())
+            b.push(synth.gradient(N, l, step, 1e-2, synth.GRAD_BF16, seed=2), b.gpu.timestamp())
+        assert a.gpu.step() == 1 and b.gpu.step() == 1
+        assert a.cpu.step() == 1 and b.cpu.step() == 1
+    a.gpu.sync(), b.gpu.sync()
+    a._alive.clear(), b._alive.clear()
+    a.compare(REL_100_STEPS)
+    b.compare(REL_100_STEPS)
+    a.close(), b.close()
+
+
+def test_queue_capacity_is_reported():
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    ps = rb.ParameterServer(64, 128, 1, 0.1)     # c = 128: nothing steps while we fill the queue
+    g = torch.zeros(64, device="cuda")
+    for i in range(rb.QUEUE_CAP):
+        assert ps.push(g, 0) == i + 1
+    with pytest.raises(rb.RudraError) as e:
+        ps.push(g, 0)
+    assert e.value.code == rb.E_QUEUE_FULL
+    done = 0
+    while ps.step() == 1:
+        done += 1
+    assert done == rb.QUEUE_CAP // 128 and ps.timestamp() == done
+    ps.close()
