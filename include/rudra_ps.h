@@ -159,9 +159,34 @@ int rudra_ps_import_state(rudra_ps* ps, const float* theta_src_dev, const float*
  * errors as RUDRA_E_CUDA. */
 int rudra_ps_sync(rudra_ps* ps);
 
-/* Counters since create: out[0] pushes, out[1] updates, out[2] pulls served (destinations),
- * out[3] kernels launched, out[4] bytes copied host->device, out[5] bytes copied device->host. */
-int rudra_ps_counters(const rudra_ps* ps, uint64_t out[6]);
+/* Counters since create: out[0] pushes, out[1] updates, out[2] pulls served (learners),
+ * out[3] kernels launched, out[4] bytes copied host->device, out[5] bytes copied device->host,
+ * out[6] copies of the weights written for pulls, out[7] of those, shared versions (zero-copy). */
+int rudra_ps_counters(const rudra_ps* ps, uint64_t out[8]);
+
+/*
+ * Zero-copy pulls.  Section 3.3 gives each learner a computation buffer and a communication
+ * buffer for pullWeights, so that using newly received weights "only requires a pointer swap".
+ * With learners and server sharing one GPU's memory the same idea removes the copy: the handle
+ * keeps a pool of nversions immutable weight vectors, a pull hands the learner a pointer to the
+ * one holding the current timestamp, and learners that pull the same timestamp share it -- a
+ * version is written once (4 bytes per weight, by the update kernel when the pull sits in a
+ * rudra_ps_run_events batch) however many learners read it.
+ *
+ * rudra_ps_enable_views allocates the pool (nparams floats each; legal only while no learner holds
+ * a view).  rudra_ps_pull_view gives learner `learner` (0 <= learner < lambda) the current
+ * version and takes back the one it held; returns the timestamp and stores the device pointer in
+ * *view_out.  The pointer stays valid, and the vector behind it unchanged, until the same
+ * learner's next pull; the learner must have finished reading the old vector (ordered before the
+ * handle's stream) when it makes that call.  If every version is still held by some learner the
+ * call fails with RUDRA_E_STATE and nothing changes: lambda + 1 versions always suffice.
+ * While views are enabled, the PULL and BROADCAST events of rudra_ps_run_events are served this
+ * way (slots_dev is ignored; BROADCAST hands the current version to all lambda learners) and
+ * rudra_ps_view_of reads back a learner's current view and its timestamp.
+ */
+int rudra_ps_enable_views(rudra_ps* ps, uint32_t nversions);
+int64_t rudra_ps_pull_view(rudra_ps* ps, uint32_t learner, const float** view_out);
+int64_t rudra_ps_view_of(const rudra_ps* ps, uint32_t learner, const float** view_out);
 
 /* Reason of the calling thread's most recent failure; static storage, never freed. */
 const char* rudra_last_error(void);

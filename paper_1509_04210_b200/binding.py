@@ -83,6 +83,9 @@ def lib():
         "rudra_sched_destroy": (None, [vp]),
         "rudra_sched_next": (i64, [vp, vp, u64]),
         "rudra_ps_run_events": (i64, [vp, vp, u64, vp, vp, u32]),
+        "rudra_ps_enable_views": (C.c_int, [vp, u32]),
+        "rudra_ps_pull_view": (i64, [vp, u32, vp]),
+        "rudra_ps_view_of": (i64, [vp, u32, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -245,9 +248,24 @@ class ParameterServer:
         _check(lib().rudra_ps_sync(self._h))
 
     def counters(self):
-        out = np.zeros(6, dtype=np.uint64)
+        out = np.zeros(8, dtype=np.uint64)
         _check(lib().rudra_ps_counters(self._h, out.ctypes.data))
-        return dict(zip(("pushes", "updates", "pulls", "launches", "h2d_bytes", "d2h_bytes"), (int(x) for x in out)))
+        names = ("pushes", "updates", "pulls", "launches", "h2d_bytes", "d2h_bytes", "weight_copies", "versions")
+        return dict(zip(names, (int(x) for x in out)))
+
+    def enable_views(self, nversions):
+        _check(lib().rudra_ps_enable_views(self._h, int(nversions)))
+
+    def pull_view(self, learner):
+        """(device address of the learner's new read-only weight vector, its timestamp)."""
+        ptr = C.c_void_p(0)
+        ts = _check(lib().rudra_ps_pull_view(self._h, int(learner), C.byref(ptr)))
+        return ptr.value, ts
+
+    def view_of(self, learner):
+        ptr = C.c_void_p(0)
+        ts = _check(lib().rudra_ps_view_of(self._h, int(learner), C.byref(ptr)))
+        return ptr.value, ts
 
     def close(self):
         if getattr(self, "_h", None):

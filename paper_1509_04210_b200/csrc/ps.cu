@@ -89,7 +89,15 @@ struct rudra_ps {
   std::vector<uint32_t> sigma;
   std::vector<float> scale;
   double avg_sigma = 0.0;
-  uint64_t counters[6] = {0, 0, 0, 0, 0, 0};
+  uint64_t counters[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+
+  // Zero-copy pulls (rudra_ps_enable_views): a pool of immutable weight versions.  A pull hands
+  // the learner a pointer to the version with the current timestamp; learners that pull the same
+  // timestamp share one buffer, so a version is written once however many learners read it.
+  struct Version { float* buf = nullptr; uint64_t ts = 0; uint32_t refs = 0; bool valid = false; };
+  std::vector<Version> versions;
+  std::vector<int> view_of;        // per learner: index into versions, or -1
+  bool views_enabled() const { return !versions.empty(); }
 
   size_t grad_bytes() const { return (size_t)N * (gtype == RUDRA_GRAD_BF16 ? 2u : 4u); }
 };
@@ -163,7 +171,46 @@ int check_push(rudra_ps* ps, uint64_t pulled_ts) {
 struct Window {
   rudra::UpdateParams p;
   uint32_t nupd = 0, ndst = 0;
+  uint32_t npulls = 0;           // learner pulls served (a shared version serves several with one copy)
+  uint32_t nversions = 0;        // versions written by this launch
   std::vector<int> used_slots;   // staging slots the window's gradients occupy
+};
+
+// Bookkeeping of the version pool, separate from the device buffers so that a batch can be
+// replayed on a copy before anything is launched.
+struct ViewBook {
+  std::vector<uint64_t> ts;
+  std::vector<uint32_t> refs;
+  std::vector<uint8_t> valid;
+  std::vector<int> view_of;
+
+  explicit ViewBook(const rudra_ps* ps) : view_of(ps->view_of) {
+    for (const auto& v : ps->versions) { ts.push_back(v.ts); refs.push_back(v.refs); valid.push_back(v.valid); }
+  }
+  // Learner l takes the version with timestamp now.  Returns its index, sets *fresh when the
+  // version has to be written first; -1 when every buffer is still held by some learner.
+  int adopt(uint32_t l, uint64_t now, bool* fresh) {
+    *fresh = false;
+    int idx = -1;
+    for (size_t i = 0; i < ts.size(); ++i)
+      if (valid[i] && ts[i] == now) { idx = (int)i; break; }
+    if (idx < 0) {
+      const int own = view_of[l];   // the learner's own old version becomes free with this pull
+      for (size_t i = 0; i < ts.size(); ++i)
+        if (refs[i] == 0 || ((int)i == own && refs[i] == 1)) { idx = (int)i; break; }
+      if (idx < 0) return -1;
+      *fresh = true;
+    }
+    if (view_of[l] >= 0) refs[view_of[l]] -= 1;
+    if (*fresh) { ts[idx] = now; valid[idx] = 1; }
+    refs[idx] += 1;
+    view_of[l] = idx;
+    return idx;
+  }
+  void store(rudra_ps* ps) const {
+    for (size_t i = 0; i < ts.size(); ++i) { ps->versions[i].ts = ts[i]; ps->versions[i].refs = refs[i]; ps->versions[i].valid = valid[i] != 0; }
+    ps->view_of = view_of;
+  }
 };
 
 // Group close (Section 3.1, Eq. 2) and the step-size table (Eq. 5's 1/c times the rate of Eq. 6
@@ -219,7 +266,11 @@ bool window_has_room_for_update(const rudra_ps* ps, const Window& w, uint32_t ma
 
 // Enqueues the window: the fused kernel if it holds updates, a plain snapshot if it holds only pulls.
 int flush_window(rudra_ps* ps, Window& w) {
-  if (w.nupd == 0 && w.ndst == 0) return 0;
+  if (w.nupd == 0 && w.ndst == 0) {   // nothing to launch; pulls may still have been served by sharing
+    ps->counters[2] += w.npulls;
+    w.npulls = 0;
+    return 0;
+  }
   cudaError_t e;
   if (w.nupd == 0) {
     rudra::SnapshotParams sp;
@@ -249,10 +300,12 @@ int flush_window(rudra_ps* ps, Window& w) {
     ps->free_slots.push_back(slot);
   }
   ps->counters[1] += w.nupd;
-  ps->counters[2] += w.ndst;
+  ps->counters[2] += w.npulls;
   ps->counters[3] += 1;
+  ps->counters[6] += w.ndst;
+  ps->counters[7] += w.nversions;
   w.used_slots.clear();
-  w.nupd = w.ndst = 0;
+  w.nupd = w.ndst = w.npulls = w.nversions = 0;
   if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
   return 0;
 }
@@ -269,6 +322,7 @@ int do_step(rudra_ps* ps, float* const* dsts, uint32_t k) {
   Window w;
   append_update(ps, w);
   for (uint32_t d = 0; d < k; ++d) w.p.dst[w.ndst++] = dsts[d];
+  w.npulls = k;
   if (int r = flush_window(ps, w)) return r;
   return 1;
 }
@@ -320,6 +374,7 @@ void rudra_ps_destroy(rudra_ps* ps) {
   if (!valid(ps)) return;
   DeviceScope dev(ps->device);
   free_host_path(ps);
+  for (auto& v : ps->versions) cudaFree(v.buf);
   cudaFree(ps->theta);
   cudaFree(ps->state);
   ps->magic = 0;
@@ -380,6 +435,7 @@ static int set_weights_common(rudra_ps* ps, const float* src, cudaMemcpyKind kin
   release_queue(ps);
   ps->ts = 0;
   ps->has_clock = false;
+  for (auto& v : ps->versions) v.valid = false;   // held views keep their contents; none matches the new weights
   return 0;
 }
 
@@ -446,9 +502,12 @@ int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t co
   if (count && !events) return fail(RUDRA_E_INVAL, "null event list");
   const uint32_t cap = max_window == 0 || max_window > (uint32_t)rudra::kMaxWindow ? (uint32_t)rudra::kMaxWindow : max_window;
   // Pass 1: replay the integers only.  Nothing is queued or launched unless the whole batch is legal.
+  const bool views = ps->views_enabled();
   {
     uint64_t ts = ps->ts;
     uint64_t queued = ps->queue.size();
+    ViewBook sim(ps);
+    bool fresh;
     for (uint64_t i = 0; i < count; ++i) {
       const rudra_event& ev = events[i];
       const bool needs_learner = ev.kind == RUDRA_EV_PUSH || ev.kind == RUDRA_EV_PULL;
@@ -467,12 +526,21 @@ int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t co
           if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: update expects new timestamp %llu, server reaches %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
           break;
         case RUDRA_EV_PULL:
-          if (!slots_dev || !aligned(slots_dev[ev.learner])) return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
           if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: pull expects timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+          if (views) {
+            if (sim.adopt(ev.learner, ts, &fresh) < 0) return fail(RUDRA_E_STATE, "event %llu: all %zu weight versions are still held by learners", (unsigned long long)i, sim.ts.size());
+          } else if (!slots_dev || !aligned(slots_dev[ev.learner])) {
+            return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
+          }
           break;
         case RUDRA_EV_PULL_SKIP:
           break;
         case RUDRA_EV_BROADCAST:
+          if (views) {
+            for (uint32_t l = 0; l < ps->lambda; ++l)
+              if (sim.adopt(l, ts, &fresh) < 0) return fail(RUDRA_E_STATE, "event %llu: all %zu weight versions are still held by learners", (unsigned long long)i, sim.ts.size());
+            break;
+          }
           if (!slots_dev) return fail(RUDRA_E_INVAL, "event %llu: broadcast without slots", (unsigned long long)i);
           for (uint32_t l = 0; l < ps->lambda; ++l)
             if (!aligned(slots_dev[l])) return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, l);
@@ -488,10 +556,24 @@ int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t co
   if (!dev.ok()) return fail(RUDRA_E_CUDA, "cannot select device %d", ps->device);
   Window w;
   int64_t updates = 0;
-  auto add_pull = [&](float* dst) -> int {
+  ViewBook book(ps);
+  auto add_copy = [&](float* dst) -> int {
     if (w.ndst == (uint32_t)rudra::kMaxDsts)
       if (int r = flush_window(ps, w)) return r;
     w.p.dst[w.ndst++] = dst;
+    return 0;
+  };
+  // One learner's pull: a copy into its slot, or (zero-copy mode) a reference to the version with
+  // the current timestamp, which is written at most once however many learners take it.
+  auto add_pull = [&](uint32_t learner) -> int {
+    w.npulls += 1;
+    if (!views) return add_copy(slots_dev[learner]);
+    bool fresh = false;
+    const int idx = book.adopt(learner, ps->ts, &fresh);
+    if (fresh) {
+      if (int r = add_copy(ps->versions[idx].buf)) return r;
+      w.nversions += 1;
+    }
     return 0;
   };
   for (uint64_t i = 0; i < count; ++i) {
@@ -507,18 +589,73 @@ int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t co
         updates += 1;
         break;
       case RUDRA_EV_PULL:
-        if (int r = add_pull(slots_dev[ev.learner])) return r;
+        if (int r = add_pull(ev.learner)) return r;
         break;
       case RUDRA_EV_BROADCAST:
         for (uint32_t l = 0; l < ps->lambda; ++l)
-          if (int r = add_pull(slots_dev[l])) return r;
+          if (int r = add_pull(l)) return r;
         break;
       default:
         break;
     }
   }
+  if (views) book.store(ps);
   if (int r = flush_window(ps, w)) return r;
   return updates;
+}
+
+int rudra_ps_enable_views(rudra_ps* ps, uint32_t nversions) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (nversions < 2 || nversions > 4096) return fail(RUDRA_E_INVAL, "need 2 <= nversions <= 4096");
+  for (int v : ps->view_of)
+    if (v >= 0) return fail(RUDRA_E_STATE, "learners still hold views");
+  DeviceScope dev(ps->device);
+  cudaError_t e = cudaStreamSynchronize(ps->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  for (auto& v : ps->versions) cudaFree(v.buf);
+  ps->versions.clear();
+  ps->view_of.assign(ps->lambda, -1);
+  for (uint32_t i = 0; i < nversions; ++i) {
+    rudra_ps::Version v;
+    e = cudaMalloc(reinterpret_cast<void**>(&v.buf), ps->N * sizeof(float));
+    if (e != cudaSuccess) {
+      for (auto& u : ps->versions) cudaFree(u.buf);
+      ps->versions.clear();
+      return cuda_fail(e, "weight version allocation");
+    }
+    ps->versions.push_back(v);
+  }
+  return 0;
+}
+
+int64_t rudra_ps_pull_view(rudra_ps* ps, uint32_t learner, const float** view_out) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!ps->views_enabled()) return fail(RUDRA_E_STATE, "call rudra_ps_enable_views first");
+  if (learner >= ps->lambda || !view_out) return fail(RUDRA_E_INVAL, "learner out of range or null output");
+  ViewBook book(ps);
+  bool fresh = false;
+  const int idx = book.adopt(learner, ps->ts, &fresh);
+  if (idx < 0) return fail(RUDRA_E_STATE, "all %zu weight versions are still held by learners", ps->versions.size());
+  DeviceScope dev(ps->device);
+  Window w;
+  w.npulls = 1;
+  if (fresh) {
+    w.p.dst[w.ndst++] = ps->versions[idx].buf;
+    w.nversions = 1;
+  }
+  book.store(ps);
+  if (int r = flush_window(ps, w)) return r;   // a snapshot launch if the version is new
+  *view_out = ps->versions[idx].buf;
+  return (int64_t)ps->ts;
+}
+
+int64_t rudra_ps_view_of(const rudra_ps* ps, uint32_t learner, const float** view_out) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  if (!ps->views_enabled() || learner >= ps->lambda || !view_out) return fail(RUDRA_E_INVAL, "views not enabled, learner out of range or null output");
+  const int idx = ps->view_of[learner];
+  if (idx < 0) return fail(RUDRA_E_STATE, "learner %u holds no view", learner);
+  *view_out = ps->versions[idx].buf;
+  return (int64_t)ps->versions[idx].ts;
 }
 
 int64_t rudra_ps_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) {
@@ -540,6 +677,7 @@ int64_t rudra_ps_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) {
   if (e != cudaSuccess) return cuda_fail(e, "snapshot kernel launch");
   ps->counters[2] += k;
   ps->counters[3] += 1;
+  ps->counters[6] += k;
   return (int64_t)ps->ts;
 }
 
@@ -583,6 +721,7 @@ int64_t rudra_ps_pull_host(rudra_ps* ps, float* dst_host) {
   ps->counters[2] += 1;
   ps->counters[3] += 1;
   ps->counters[5] += ps->N * sizeof(float);
+  ps->counters[6] += 1;
   return (int64_t)ps->ts;
 }
 
@@ -626,6 +765,7 @@ int rudra_ps_import_state(rudra_ps* ps, const float* theta_src_dev, const float*
   release_queue(ps);
   ps->ts = ts;
   ps->has_clock = false;
+  for (auto& v : ps->versions) v.valid = false;
   return 0;
 }
 
@@ -637,7 +777,7 @@ int rudra_ps_sync(rudra_ps* ps) {
   return 0;
 }
 
-int rudra_ps_counters(const rudra_ps* ps, uint64_t out[6]) {
+int rudra_ps_counters(const rudra_ps* ps, uint64_t out[8]) {
   if (!valid(ps) || !out) return fail(RUDRA_E_INVAL, "bad handle or null output");
   std::memcpy(out, ps->counters, sizeof(ps->counters));
   return 0;
