@@ -120,21 +120,23 @@ def launches_in_region(ps, c0):
     return ps.counters()["launches"] - c0["launches"]
 
 
-def default_window(w):
+def default_window(w, views=False):
     """Updates packed into one launch by default: the gradients lambda learners can have waiting at
     once make n = lambda / c updates (every learner blocks on its push until the server has taken
-    it), capped by the launch tables (32 updates, 128 gradients, 128 pull destinations)."""
-    pulls_per_update = w.lam if (w.downcast or w.mode == synth.HARDSYNC) else w.c
+    it), capped by the launch tables (32 updates, 128 gradients, 128 pull destinations; with
+    zero-copy pulls a version is one destination however many learners take it)."""
+    pulls_per_update = 1 if views else (w.lam if (w.downcast or w.mode == synth.HARDSYNC) else w.c)
     return max(1, min(w.n, 32, 128 // w.c, 128 // pulls_per_update))
 
 
-def window_bytes_per_param(w, events):
+def window_bytes_per_param(w, events, copies=None):
     """Algorithmic bytes per weight of one launch over these events: every gradient read once,
-    weights and state read and written once, one write per pulled copy."""
+    weights and state read and written once, one write per copy of the weights handed out."""
     g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
     pushes = int((events["kind"] == EV_STEP).sum()) * w.c
-    pulls = int((events["kind"] == EV_PULL).sum()) + w.lam * int((events["kind"] == EV_BROADCAST).sum())
-    return pushes * g + state_bytes(w) + 4 * pulls
+    if copies is None:
+        copies = int((events["kind"] == EV_PULL).sum()) + w.lam * int((events["kind"] == EV_BROADCAST).sum())
+    return pushes * g + state_bytes(w) + 4 * copies
 
 
 class ClockSampler(threading.Thread):
@@ -308,19 +310,24 @@ def run_ours(args, w):
     stream = torch.cuda.Stream()
     nbufs = min(w.lam, args.buffers) if args.buffers else w.lam
     bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype, seed) for l in range(nbufs)]
-    nslots = nbufs
+    views = args.pull == "views"
+    nslots = 0 if views else nbufs
     slots = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(nslots)]
     ps = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
     ps.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
     if args.optimizer == "adagrad":
         ps.set_option(rb.OPT_OPTIMIZER, rb.OPTIM_ADAGRAD)
     ps.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
+    if views:
+        ps.enable_views(w.lam + 1)
     ps.sync()
     ps.set_stream(stream)
     windows = make_windows(w, args.warmup + args.steps)
-    W = default_window(w) if args.window < 0 else args.window
+    W = default_window(w, views) if args.window < 0 else args.window
+    if views and W == 0:
+        raise SystemExit("--pull views is served through rudra_ps_run_events: use --window >= 1")
     gtable = rb.pointer_table([bufs[l % nbufs] for l in range(w.lam)])
-    stable = rb.pointer_table([slots[l % nslots] for l in range(w.lam)])
+    stable = None if views else rb.pointer_table([slots[l % nslots] for l in range(w.lam)])
 
     def new_events():
         return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -344,10 +351,15 @@ def run_ours(args, w):
     def run_backlog(chunk, timed):
         """A backlog of W update windows through run_events: one launch when the tables allow."""
         e0, e1 = new_events()
+        copies0 = ps.counters()["weight_copies"] if views else 0
         e0.record(stream)
         ps.run_events(chunk, gtable, stable, W)
         e1.record(stream)
-        timed.append((e0, e1, window_bytes_per_param(w, chunk) * N))
+        if views:   # a version is written once however many learners pulled it
+            bpp = window_bytes_per_param(w, chunk, copies=ps.counters()["weight_copies"] - copies0)
+        else:
+            bpp = window_bytes_per_param(w, chunk)
+        timed.append((e0, e1, bpp * N))
 
     def prepare(wins):
         """The messages as the server receives them: single windows, or backlogs of W windows."""
@@ -381,6 +393,7 @@ def run_ours(args, w):
     upd_ms = kern_ms / max(len(timed), 1)
     launches = c1["launches"] - c0["launches"]
     pulls = c1["pulls"] - c0["pulls"]
+    copies = c1["weight_copies"] - c0["weight_copies"]
 
     e2e_ms, e2e_steps, h0, h1 = float('nan'), 0, None, None
     if not args.kernel_only:
@@ -444,10 +457,12 @@ def run_ours(args, w):
         if W == 0:
             path_bytes = N * (args.steps * (w.c * g + sb) + 8 * pulls)
         else:
-            path_bytes = N * (args.steps * w.c * g + launches * sb + 4 * pulls)
+            path_bytes = N * (args.steps * w.c * g + launches * sb + 4 * copies)
         value = replicas.whole_job_rate(args.steps, world, ms)
         cfg = workload_config(w)
         cfg["window"] = W
+        cfg["pull"] = ("zero-copy: learners share a pointer to the version they pulled (rudra_ps_enable_views)" if views
+                       else "copy into each learner's slot")
         cfg["window_note"] = ("messages handled one at a time (push / step / pull)" if W == 0 else
                               "backlog of %d update windows per rudra_ps_run_events call" % W)
         line = {
@@ -458,6 +473,7 @@ def run_ours(args, w):
             "hbm_gbs_whole_path": path_bytes / (ms * 1e-3) / 1e9,
             "bytes_per_param_per_step": path_bytes / N / args.steps,
             "pulls_per_step": pulls / args.steps,
+            "weight_copies_per_step": copies / args.steps,
             "gpu_launches": launches,
             "clocks": clocks,
             "e2e": None if args.kernel_only else {
@@ -507,6 +523,8 @@ def main():
     ap.add_argument("--window", type=int, default=-1,
                     help="update windows handed to the server per call: 0 = one message at a time, "
                          "-1 = what lambda blocked learners can have waiting (n = lambda/c updates)")
+    ap.add_argument("--pull", default="copy", choices=["copy", "views"],
+                    help="copy: every pull writes the learner's own slot; views: zero-copy shared weight versions")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adagrad"],
                     help="momentum SGD with weight decay (Section 4.2) or AdaGrad at the server (Section 5.5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -525,6 +543,12 @@ def main():
         global ADAGRAD
         ADAGRAD = True
         w = dataclasses.replace(w, name=w.name + "+adagrad", momentum=0.0)
+    if args.pull == "views" and w.downcast:
+        import dataclasses
+
+        # with shared versions the down-cast needs no broadcast: each learner takes the current
+        # version when it starts its next mini-batch (the integers of the trace are the same)
+        w = dataclasses.replace(w, name=w.name + "+views", downcast=False)
     if args.nparams:
         import dataclasses
 
