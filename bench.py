@@ -129,16 +129,6 @@ def default_window(w, views=False):
     return max(1, min(w.n, 32, 128 // w.c, 128 // pulls_per_update))
 
 
-def window_bytes_per_param(w, events, copies=None):
-    """Algorithmic bytes per weight of one launch over these events: every gradient read once,
-    weights and state read and written once, one write per copy of the weights handed out."""
-    g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
-    pushes = int((events["kind"] == EV_STEP).sum()) * w.c
-    if copies is None:
-        copies = int((events["kind"] == EV_PULL).sum()) + w.lam * int((events["kind"] == EV_BROADCAST).sum())
-    return pushes * g + state_bytes(w) + 4 * copies
-
-
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons while the timed region runs (read-only NVML queries)."""
 
@@ -329,8 +319,21 @@ def run_ours(args, w):
     gtable = rb.pointer_table([bufs[l % nbufs] for l in range(w.lam)])
     stable = None if views else rb.pointer_table([slots[l % nslots] for l in range(w.lam)])
 
+    event_pool = []
+
     def new_events():
+        """A pair of timing events; pairs made before the timed region are re-used inside it so that
+        no event is created between launches."""
+        if event_pool:
+            return event_pool.pop()
         return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def fill_event_pool(count):
+        for _ in range(count):
+            pair = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            pair[0].record(stream)      # the first record creates the underlying event
+            pair[1].record(stream)
+            event_pool.append(pair)
 
     def run_messages(win, timed):
         """One message at a time through push / step / pull (--window 0)."""
@@ -342,7 +345,7 @@ def run_ours(args, w):
                 e0.record(stream)
                 ps.step()
                 e1.record(stream)
-                timed.append((e0, e1, update_bytes_per_param(w) * N))
+                timed.append((e0, e1))
             elif kind == EV_PULL:
                 ps.pull(slots[learner % nslots])
             elif kind == EV_BROADCAST:
@@ -351,15 +354,10 @@ def run_ours(args, w):
     def run_backlog(chunk, timed):
         """A backlog of W update windows through run_events: one launch when the tables allow."""
         e0, e1 = new_events()
-        copies0 = ps.counters()["weight_copies"] if views else 0
         e0.record(stream)
         ps.run_events(chunk, gtable, stable, W)
         e1.record(stream)
-        if views:   # a version is written once however many learners pulled it
-            bpp = window_bytes_per_param(w, chunk, copies=ps.counters()["weight_copies"] - copies0)
-        else:
-            bpp = window_bytes_per_param(w, chunk)
-        timed.append((e0, e1, bpp * N))
+        timed.append((e0, e1))
 
     def prepare(wins):
         """The messages as the server receives them: single windows, or backlogs of W windows."""
@@ -373,6 +371,7 @@ def run_ours(args, w):
 
     warm_batches, timed_batches = prepare(windows[: args.warmup]), prepare(windows[args.warmup:])
     run_all(warm_batches, [])
+    fill_event_pool(args.steps + 2 if W == 0 else len(timed_batches) + 2)
     barrier()
     sampler = ClockSampler(visible_gpu_index(local_rank))
     sampler.start()
@@ -388,8 +387,7 @@ def run_ours(args, w):
     ms = start.elapsed_time(end)
     if W != 0 and launches_in_region(ps, c0) != len(timed):
         timed = []      # a backlog needed more than one launch: no per-launch figure for this shape
-    kern_ms = float(sum(a.elapsed_time(b) for a, b, _ in timed))
-    kern_bytes = float(sum(nb for _, _, nb in timed))
+    kern_ms = float(sum(a.elapsed_time(b) for a, b in timed))
     upd_ms = kern_ms / max(len(timed), 1)
     launches = c1["launches"] - c0["launches"]
     pulls = c1["pulls"] - c0["pulls"]
@@ -451,13 +449,16 @@ def run_ours(args, w):
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
         g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
-        achieved = kern_bytes / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else float("nan")
         # bytes the whole path must move per step: every gradient once, weights/state per launch, pulls
         sb = state_bytes(w)
         if W == 0:
             path_bytes = N * (args.steps * (w.c * g + sb) + 8 * pulls)
         else:
             path_bytes = N * (args.steps * w.c * g + launches * sb + 4 * copies)
+        # the timed launches: with a backlog every launch of the region (so their bytes are the whole
+        # path's), one message at a time only the update kernels
+        kern_bytes = float(path_bytes if W != 0 else N * args.steps * (w.c * g + sb))
+        achieved = kern_bytes / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else float("nan")
         value = replicas.whole_job_rate(args.steps, world, ms)
         cfg = workload_config(w)
         cfg["window"] = W

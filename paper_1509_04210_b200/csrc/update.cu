@@ -28,6 +28,7 @@ namespace rudra {
 namespace {
 
 constexpr int kUnit = 8;   // weights per thread per unit
+constexpr uint64_t kSmallModel = 262144;   // below this many weights the one-weight-per-thread kernel runs
 
 struct alignas(32) F8 { float v[kUnit]; };
 
@@ -222,6 +223,60 @@ __global__ void __launch_bounds__(THREADS) update_kernel(const __grid_constant__
   }
 }
 
+// Small models (a few hundred thousand weights and fewer: the paper's CIFAR10 network has ~90 K)
+// are not bandwidth-bound but latency-bound: with 8 weights per thread there are only a handful of
+// warps per SM and every instruction's latency shows.  This variant gives every weight its own
+// thread (coalesced 4-byte accesses) and keeps DEPTH gradient loads in flight; the arithmetic and
+// its order are those of the kernel above.
+template <typename G, int OPT, bool STATE, int DEPTH, int THREADS>
+__global__ void __launch_bounds__(THREADS) update_kernel_small(const __grid_constant__ UpdateParams p) {
+  const uint64_t k = (uint64_t)blockIdx.x * THREADS + threadIdx.x;
+  if (k >= p.n) return;
+  float th = p.theta[k];
+  float st = STATE ? p.state[k] : 0.f;
+  uint32_t d = 0;
+  for (const uint32_t d1 = p.dst_end[0]; d < d1; ++d) p.dst[d][k] = th;
+  const uint32_t total = p.nupd * p.c;
+  uint32_t w = 0, left = p.c;
+  float acc = 0.f;
+  for (uint32_t l0 = 0; l0 < total; l0 += DEPTH) {
+    float g[DEPTH];
+#pragma unroll
+    for (int i = 0; i < DEPTH; ++i)
+      if (l0 + i < total) g[i] = GradUnit<G>::scalar(p.grad[l0 + i], k);
+#pragma unroll
+    for (int i = 0; i < DEPTH; ++i) {
+      if (l0 + i < total) {
+        acc = fmaf(p.scale[l0 + i], g[i], acc);
+        if (--left == 0) {
+          apply<OPT, STATE>(p, p.awd[w], p.abar[w], acc, th, st);
+          acc = 0.f;
+          ++w;
+          left = p.c;
+          for (const uint32_t d1 = p.dst_end[w]; d < d1; ++d) p.dst[d][k] = th;
+        }
+      }
+    }
+  }
+  p.theta[k] = th;
+  if (STATE) p.state[k] = st;
+}
+
+template <typename G, int OPT, bool STATE>
+cudaError_t launch_small(const UpdateParams& p, cudaStream_t stream) {
+  constexpr int THREADS = 128, DEPTH = 8;
+  const uint64_t blocks = (p.n + THREADS - 1) / THREADS;
+  update_kernel_small<G, OPT, STATE, DEPTH, THREADS><<<(unsigned)blocks, THREADS, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename G>
+cudaError_t launch_small_typed(const UpdateParams& p, Optim optim, cudaStream_t stream) {
+  if (optim == kAdagrad) return launch_small<G, kAdagrad, true>(p, stream);
+  if (p.momentum != 0.f) return launch_small<G, kMomentumSgd, true>(p, stream);
+  return launch_small<G, kMomentumSgd, false>(p, stream);
+}
+
 template <typename G, int OPT, bool STATE, int DEPTH, int U, int THREADS>
 cudaError_t launch_one(const UpdateParams& p, cudaStream_t stream) {
   const uint64_t nunits = p.n / kUnit;
@@ -242,6 +297,8 @@ cudaError_t launch_typed(const UpdateParams& p, Optim optim, cudaStream_t stream
 }  // namespace
 
 cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, cudaStream_t stream) {
+  if (p.n < kSmallModel)   // latency-bound: one weight per thread
+    return gtype == kBF16 ? launch_small_typed<__nv_bfloat16>(p, optim, stream) : launch_small_typed<float>(p, optim, stream);
   // Large vectors: 256-thread tiles (measured: any tile shape saturates HBM).  Vectors that give
   // fewer than ~16 such tiles per SM of a 148-SM part are latency-bound or leave the last wave
   // ragged: 64-thread tiles spread them over four times as many blocks.

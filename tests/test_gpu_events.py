@@ -59,6 +59,8 @@ CASES = [
     ("mid", 30005, 900, 0),
     ("imagenet", 40001, 1200, 0),
     ("imagenet", 40001, 1200, 5),
+    ("imagenet", 300011, 700, 0),
+    ("mid", 262144 + 3, 500, 0),
     ("stress", 9001, 1500, 0),
     ("stress", 9001, 1500, 1),
 ]

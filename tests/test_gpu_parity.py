@@ -51,6 +51,9 @@ def test_stress_shape_small_bf16_downcast():
 
 
 SIZES = [1, 3, 7, 8, 9, 15, 2047, 2048, 2049, 4096 + 5, 8 * 256 * 3 + 1, 8 * 256 * 2 * 5 + 13, 300007]
+# lengths at and above 262 144 weights run the 8-weights-per-thread kernel (ragged tiles and tails),
+# shorter ones the one-weight-per-thread kernel for small models
+VECTOR_SIZES = [262144, 262144 + 1, 262144 + 7, 262144 + 8 * 64 + 9, 262144 + 8 * 256 * 3 + 5, 300007]
 GROUPS = [1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 64, 128]
 
 
@@ -59,7 +62,7 @@ def test_sizes_and_group_widths(dtype):
     # ragged vector lengths x group widths around every unroll boundary of the kernels
     rng = np.random.default_rng(5)
     for i, c in enumerate(GROUPS):
-        for N in (SIZES[i % len(SIZES)], SIZES[(3 * i + 1) % len(SIZES)], SIZES[-1] if c in (3, 32) else 9):
+        for N in (SIZES[i % len(SIZES)], SIZES[(3 * i + 1) % len(SIZES)], VECTOR_SIZES[i % len(VECTOR_SIZES)]):
             pair = Pair(N, c, 1, 0.05, 0.9, 5e-4, dtype, policy=ora.LR_PER_GRADIENT, seed=100 + i)
             for step in range(2):
                 for l in range(c):
@@ -88,13 +91,14 @@ def test_adagrad_parity():
     pair.close()
 
 
+@pytest.mark.parametrize("N", [70003, 300011])
 @pytest.mark.parametrize("dtype,optimizer", [(synth.GRAD_F32, ora.OPT_MOMENTUM_SGD), (synth.GRAD_BF16, ora.OPT_MOMENTUM_SGD),
                                              (synth.GRAD_F32, ora.OPT_ADAGRAD)])
-def test_bit_exact_against_the_fp32_evaluation_of_the_oracle(dtype, optimizer):
+def test_bit_exact_against_the_fp32_evaluation_of_the_oracle(dtype, optimizer, N):
     # Not the parity bar (that is the double-precision oracle, above) but a sharper net: the kernel
     # has no cross-thread reduction, so with the oracle evaluating the same rule in fp32, one fma
     # per term in arrival order, every weight and state value must agree to the last bit.
-    N, lam, n = 70003, 15, 3
+    lam, n = 15, 3
     pair = Pair(N, lam, n, 0.03, 0.9 if optimizer == ora.OPT_MOMENTUM_SGD else 0.0, 5e-4, dtype,
                 policy=ora.LR_PER_GRADIENT, optimizer=optimizer)
     pair.cpu.set_strict(True)
@@ -132,10 +136,10 @@ def test_pull_variants_are_exact_copies():
     pair.close()
 
 
-def test_canaries_around_learner_buffers_survive():
+@pytest.mark.parametrize("N", [100003, 300003])
+def test_canaries_around_learner_buffers_survive(N):
     import torch
 
-    N = 100003
     pair = Pair(N, 2, 1, 0.1, 0.9, 0.0)
     big = torch.full((N + 64,), -123.0, device="cuda")
     dst = big[32:32 + N]

@@ -40,7 +40,7 @@ def _servers(w, N, nversions):
     return rb, out[0], out[1], grads, slots
 
 
-@pytest.mark.parametrize("name,N,nevents", [("imagenet", 30011, 1500), ("cifar10", 9001, 900), ("mid", 20003, 1200),
+@pytest.mark.parametrize("name,N,nevents", [("imagenet", 30011, 1500), ("imagenet", 280003, 600), ("cifar10", 9001, 900), ("mid", 20003, 1200),
                                             ("tiny", 4099, 300)])
 def test_views_equal_copied_slots(name, N, nevents):
     w = synth.WORKLOADS[name]
