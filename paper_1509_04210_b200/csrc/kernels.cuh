@@ -49,7 +49,8 @@ struct SnapshotParams {
 };
 
 // Enqueue one window of fused updates (and their pulls) on stream.  Returns the CUDA status of the launch.
-cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, cudaStream_t stream);
+// sm_count: multiprocessors of the device the stream belongs to (0 = unknown).
+cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, int sm_count, cudaStream_t stream);
 
 // Enqueue one 1 -> ndst copy of the weights.
 cudaError_t launch_snapshot(const SnapshotParams& p, cudaStream_t stream);

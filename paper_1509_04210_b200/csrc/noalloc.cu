@@ -112,7 +112,7 @@ int rudra_ps_update_host_noalloc(float* theta_dev, float* state_dev, uint64_t np
   p.wd = weight_decay;
   p.eps = 0.f;
   p.reverse = 0;
-  e = rudra::launch_update(p, rudra::kF32, rudra::kMomentumSgd, stream);
+  e = rudra::launch_update(p, rudra::kF32, rudra::kMomentumSgd, 0, stream);
   if (e != cudaSuccess) return fail(RUDRA_E_CUDA, cudaGetErrorString(e));
   return 0;
 }

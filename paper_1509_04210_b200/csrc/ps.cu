@@ -67,6 +67,7 @@ struct rudra_ps {
   float alpha0 = 0.f, momentum = 0.f, wd = 0.f, eps = 1e-8f;
   int gtype = RUDRA_GRAD_F32, policy = RUDRA_LR_PAPER_N, optim = RUDRA_OPTIM_MOMENTUM_SGD;
   int device = 0;
+  int sm_count = 0;
   uint32_t sweep = 0;              // launches so far: successive launches sweep in opposite directions
   cudaStream_t stream = nullptr;
   float* theta = nullptr;
@@ -271,18 +272,33 @@ int flush_window(rudra_ps* ps, Window& w) {
     w.npulls = 0;
     return 0;
   }
-  cudaError_t e;
-  if (w.nupd == 0) {
+  cudaError_t e = cudaSuccess;
+  uint32_t launches = 0;
+  auto copy_weights = [&](uint32_t d0, uint32_t d1) {   // 1 -> (d1 - d0) copy of the current weights
+    if (d1 == d0 || e != cudaSuccess) return;
     rudra::SnapshotParams sp;
-    for (uint32_t d = 0; d < w.ndst; ++d) sp.dst[d] = w.p.dst[d];
+    for (uint32_t d = d0; d < d1; ++d) sp.dst[d - d0] = w.p.dst[d];
     sp.src = ps->theta;
     sp.n = ps->N;
-    sp.ndst = w.ndst;
+    sp.ndst = d1 - d0;
     sp.reverse = ps->sweep++ & 1u;
     e = rudra::launch_snapshot(sp, ps->stream);
+    launches += 1;
+  };
+  if (w.nupd == 0) {
+    copy_weights(0, w.ndst);
   } else {
     rudra::UpdateParams& p = w.p;
     p.dst_end[w.nupd] = (uint8_t)w.ndst;
+    // A single update with a broadcast to dozens of learners around it is faster as separate
+    // launches (measured at 61 M weights, bf16, c = 32, 128 copies: 5.25 ms against 5.65 ms fused):
+    // the copies then run in the copy kernel's shape, at the price of one more read of the weights.
+    const bool split = w.nupd == 1 && w.ndst >= 64 && ps->N >= (1u << 22);
+    const uint32_t pre = p.dst_end[0], post = w.ndst;
+    if (split) {
+      copy_weights(0, pre);
+      p.dst_end[0] = p.dst_end[1] = 0;
+    }
     p.theta = ps->theta;
     p.state = ps->state;
     p.n = ps->N;
@@ -292,8 +308,13 @@ int flush_window(rudra_ps* ps, Window& w) {
     p.wd = ps->wd;
     p.eps = ps->eps;
     p.reverse = ps->sweep++ & 1u;
-    e = rudra::launch_update(p, ps->gtype == RUDRA_GRAD_BF16 ? rudra::kBF16 : rudra::kF32,
-                             ps->optim == RUDRA_OPTIM_ADAGRAD ? rudra::kAdagrad : rudra::kMomentumSgd, ps->stream);
+    if (e == cudaSuccess) {
+      e = rudra::launch_update(p, ps->gtype == RUDRA_GRAD_BF16 ? rudra::kBF16 : rudra::kF32,
+                               ps->optim == RUDRA_OPTIM_ADAGRAD ? rudra::kAdagrad : rudra::kMomentumSgd, ps->sm_count,
+                               ps->stream);
+      launches += 1;
+    }
+    if (split) copy_weights(pre, post);
   }
   for (int slot : w.used_slots) {   // the next upload into the slot waits for this launch
     cudaEventRecord(ps->slot_spent[slot], ps->stream);
@@ -301,7 +322,7 @@ int flush_window(rudra_ps* ps, Window& w) {
   }
   ps->counters[1] += w.nupd;
   ps->counters[2] += w.npulls;
-  ps->counters[3] += 1;
+  ps->counters[3] += launches;
   ps->counters[6] += w.ndst;
   ps->counters[7] += w.nversions;
   w.used_slots.clear();
@@ -354,6 +375,7 @@ rudra_ps* rudra_ps_create(uint64_t nparams, uint32_t lambda, uint32_t n, float a
   ps->N = nparams; ps->lambda = lambda; ps->n = n; ps->c = lambda / n;
   ps->alpha0 = alpha0; ps->momentum = momentum; ps->wd = weight_decay;
   cudaError_t e = cudaGetDevice(&ps->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ps->sm_count, cudaDevAttrMultiProcessorCount, ps->device);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ps->theta), nparams * sizeof(float));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ps->state), nparams * sizeof(float));
   if (e == cudaSuccess) e = cudaMemset(ps->theta, 0, nparams * sizeof(float));

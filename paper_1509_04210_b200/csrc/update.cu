@@ -296,13 +296,14 @@ cudaError_t launch_typed(const UpdateParams& p, Optim optim, cudaStream_t stream
 
 }  // namespace
 
-cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, cudaStream_t stream) {
+cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, int sm_count, cudaStream_t stream) {
   if (p.n < kSmallModel)   // latency-bound: one weight per thread
     return gtype == kBF16 ? launch_small_typed<__nv_bfloat16>(p, optim, stream) : launch_small_typed<float>(p, optim, stream);
   // Large vectors: 256-thread tiles (measured: any tile shape saturates HBM).  Vectors that give
-  // fewer than ~16 such tiles per SM of a 148-SM part are latency-bound or leave the last wave
-  // ragged: 64-thread tiles spread them over four times as many blocks.
-  const bool small = p.n / kUnit < 148ull * 16 * 256;
+  // fewer than ~16 such tiles per SM are latency-bound or leave the last wave ragged: 64-thread
+  // tiles spread them over four times as many blocks.
+  const uint64_t sms = sm_count > 0 ? (uint64_t)sm_count : 148;
+  const bool small = p.n / kUnit < sms * 16 * 256;
   if (gtype == kBF16)
     return small ? launch_typed<__nv_bfloat16, 8, 64>(p, optim, stream) : launch_typed<__nv_bfloat16, 8, 256>(p, optim, stream);
   return small ? launch_typed<float, 8, 64>(p, optim, stream) : launch_typed<float, 4, 256>(p, optim, stream);

@@ -183,3 +183,40 @@ def test_full_size_window_sampled_against_oracle():
     for s, want in last_pull.items():                            # the last writer of each slot wins
         assert rel_err(to_host(slots[s][idx_d]), want) <= REL_100_STEPS
     ps.close()
+
+
+@pytest.mark.parametrize("dtype", [synth.GRAD_F32, synth.GRAD_BF16])
+def test_broadcast_dominated_launch_equals_update_then_copies(dtype):
+    """An update that also serves 64 learner buffers is split by the library into the update and
+    a 64-way copy when the vector is large; either way it must equal the two explicit calls."""
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    N, lam, n = 5000011, 64, 2
+    c = lam // n
+    th0 = synth.device_initial_weights(N, 0.01)
+    grads = [synth.device_gradient(N, l, 1e-3, dtype) for l in range(c)]
+    out = []
+    for fused in (False, True):
+        ps = rb.ParameterServer(N, lam, n, 0.01, 0.9, 5e-4)
+        ps.set_option(rb.OPT_GRAD_DTYPE, dtype)
+        ps.set_weights(th0)
+        slots = [torch.full((N,), 3.0, device="cuda") for _ in range(lam)]
+        for step in range(2):
+            for l in range(c):
+                ps.push(grads[(l + step) % c], max(0, ps.timestamp() - (l % 2)))
+            if fused:
+                assert ps.step_pull_many(slots) == 1
+            else:
+                assert ps.step() == 1
+                assert ps.pull_many(slots) == ps.timestamp()
+        th = torch.empty(N, device="cuda")
+        st = torch.empty(N, device="cuda")
+        ps.export_state(th, st)
+        ps.sync()
+        out.append((th, st, slots))
+        ps.close()
+    (tha, sta, sa), (thb, stb, sb) = out
+    assert torch.equal(tha, thb) and torch.equal(sta, stb)
+    for i in (0, 1, 31, 63):
+        assert torch.equal(sa[i], tha) and torch.equal(sb[i], thb)
