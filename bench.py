@@ -235,7 +235,13 @@ def run_reference(args, w):
     from oracle import rudra_oracle as ora
 
     ora.build()
-    nsample = max(1, w.nparams // 4) if w.nparams > (1 << 22) else w.nparams
+    # Each step handles a bounded sample of the vector so that the whole run ends within a few
+    # minutes whatever --steps is: about 75 s of oracle work at ~60 M weight-updates per second
+    # and core, never more than a quarter of a large vector.
+    nsample = w.nparams
+    if w.nparams > (1 << 22):
+        per_step = int(75.0 * 60e6 / (args.steps + args.warmup) / max(w.c, 1) * 3)
+        nsample = max(1 << 16, min(w.nparams // 4, per_step))
     windows = make_windows(w, args.warmup + args.steps, from_oracle=True)
     grads = host_gradients(w, nsample, min(w.lam, 8))
     done, dt = oracle_run(w, windows, nsample, grads, warmup=args.warmup, adagrad=args.optimizer == "adagrad")
