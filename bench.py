@@ -387,7 +387,8 @@ def run_ours(args, w):
     clocks = sampler.stop()
     c1 = ps.counters()
     ms = start.elapsed_time(end)
-    kern_ms = float(sum(a.elapsed_time(b) for a, b in timed))
+    launch_ms = [a.elapsed_time(b) for a, b in timed]
+    kern_ms = float(sum(launch_ms))
     upd_ms = kern_ms / max(len(timed), 1)
     launches = c1["launches"] - c0["launches"]
     pulls = c1["pulls"] - c0["pulls"]
@@ -493,6 +494,10 @@ def run_ours(args, w):
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": "of %s" % peak_kind, "launches_timed": len(timed), "avg_launch_us": upd_ms * 1e3,
                 "bytes_per_launch": kern_bytes / max(len(timed), 1),
+                "launch_us": None if not launch_ms else {
+                    "min": 1e3 * min(launch_ms), "median": 1e3 * float(np.median(launch_ms)), "max": 1e3 * max(launch_ms),
+                    "first_tenth": 1e3 * float(np.mean(launch_ms[: max(1, len(launch_ms) // 10)])),
+                    "last_tenth": 1e3 * float(np.mean(launch_ms[-max(1, len(launch_ms) // 10):]))},
                 "frac_of_8TBs_datasheet": achieved / 8000.0,
                 "traffic": ncu_traffic(w.name, W, N),
             },
