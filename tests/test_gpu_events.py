@@ -220,3 +220,56 @@ def test_broadcast_dominated_launch_equals_update_then_copies(dtype):
     assert torch.equal(tha, thb) and torch.equal(sta, stb)
     for i in (0, 1, 31, 63):
         assert torch.equal(sa[i], tha) and torch.equal(sb[i], thb)
+
+
+def test_stress_config_full_size_backlog_sampled_against_oracle():
+    """The bf16, c = 32, 128-way down-cast workload at 60 965 224 weights, driven as the bench
+    drives it (one update and its broadcast per run_events call); the oracle recomputes a sample."""
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    w = synth.WORKLOADS["stress"]
+    N = w.nparams
+    rng = np.random.default_rng(4)
+    idx = np.unique(np.concatenate([np.arange(64), np.arange(N - 64, N), rng.integers(0, N, 20000)]))
+    idx_d = torch.from_numpy(idx).cuda()
+    nbuf = 40
+    bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype) for l in range(nbuf)]
+    slots = [torch.empty(N, device="cuda") for _ in range(w.lam)]
+    th0 = synth.device_initial_weights(N, w.theta_std)
+    ps = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
+    ps.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
+    ps.set_weights(th0)
+    o = ora.OraclePS(len(idx), w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
+    o.set_grad_dtype(w.grad_dtype)
+    o.set_weights(to_host(th0[idx_d]))
+    samples = [to_host(b[idx_d].view(torch.int16)).view(np.uint16) for b in bufs]
+    sched = rb.Scheduler(w.lam, w.n, w.mode, synth.MASTER_SEED, w.lognormal_sigma, w.downcast)
+    gt = [bufs[l % nbuf] for l in range(w.lam)]
+    updates = 0
+    while updates < 3:
+        ev = sched.next(1)
+        batch = [ev]
+        while ev[0]["kind"] != rb.EV_BROADCAST:       # one update window: 32 pushes, the update, the broadcast
+            ev = sched.next(1)
+            batch.append(ev)
+        batch = np.concatenate(batch)
+        assert ps.run_events(batch, gt, slots, 1) == 1
+        for e in batch:
+            if e["kind"] == ora.PUSH:
+                o.push(samples[int(e["learner"]) % nbuf], int(e["pulled_ts"]))
+            elif e["kind"] == ora.STEP:
+                assert o.step() == 1
+        updates += 1
+        th = torch.empty(N, device="cuda")
+        st = torch.empty(N, device="cuda")
+        ps.export_state(th, st)
+        ps.sync()
+        tol = 1e-5 if updates == 1 else REL_100_STEPS
+        assert rel_err(to_host(th[idx_d]), o.pull()[0]) <= tol
+        assert rel_err(to_host(st[idx_d]), o.state()) <= tol
+        np.testing.assert_array_equal(ps.last_clock()["sigma"], o.last_clock()["sigma"])
+        for i in (0, 63, 127):
+            assert torch.equal(slots[i], th)           # every learner received this version
+    assert ps.counters()["launches"] == 6             # update + 128-way copy per window
+    ps.close()
