@@ -466,6 +466,7 @@ def run_ours(args, w):
         achieved = kern_bytes / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else float("nan")
         value = replicas.whole_job_rate(args.steps, world, ms)
         cfg = workload_config(w)
+        cfg["parallelism"] = "replicas x%d (one independent server per GPU)" % world
         cfg["window"] = W
         cfg["pull"] = ("zero-copy: learners share a pointer to the version they pulled (rudra_ps_enable_views)" if views
                        else "copy into each learner's slot")
