@@ -25,6 +25,10 @@
  *     waits, flags or inter-block communication.
  *   - A handle is not thread-safe (the server of Section 3.2 handles messages one at a time);
  *     distinct handles are independent.
+ *   - Buffers named in one call must not overlap: a pull destination that aliases a queued
+ *     gradient, the weights of another handle's pending update, or another destination of a
+ *     different learner's later pull gives unspecified contents (two learners may share one slot:
+ *     the later pull wins).
  *   - There is no CPU implementation behind these calls.
  */
 #ifndef RUDRA_PS_H
