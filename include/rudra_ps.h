@@ -25,10 +25,8 @@
  *     waits, flags or inter-block communication.
  *   - A handle is not thread-safe (the server of Section 3.2 handles messages one at a time);
  *     distinct handles are independent.
- *   - Buffers named in one call must not overlap: a pull destination that aliases a queued
- *     gradient, the weights of another handle's pending update, or another destination of a
- *     different learner's later pull gives unspecified contents (two learners may share one slot:
- *     the later pull wins).
+ *   - A pull destination must not overlap a gradient buffer that is still queued; two pulls may
+ *     name the same destination, in which case the later one wins.
  *   - There is no CPU implementation behind these calls.
  */
 #ifndef RUDRA_PS_H
