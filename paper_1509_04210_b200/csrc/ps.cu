@@ -711,7 +711,7 @@ int64_t rudra_ps_pull_host(rudra_ps* ps, float* dst_host) {
   DeviceScope dev(ps->device);
   cudaError_t e = ensure_copy_streams(ps);
   if (e != cudaSuccess) return cuda_fail(e, "copy stream creation");
-  constexpr uint32_t kDownBufs = 2;
+  constexpr uint32_t kDownBufs = 4;   // snapshots that may be on their way to the host at once
   if (ps->down.size() < kDownBufs) {
     rudra_ps::DownBuf d;
     e = cudaMalloc(reinterpret_cast<void**>(&d.buf), ps->N * sizeof(float));
