@@ -152,6 +152,19 @@ int64_t rudra_ps_timestamp(const rudra_ps* ps);
 int rudra_ps_last_clock(const rudra_ps* ps, uint64_t* pulled_ts_out, uint32_t* sigma_out,
                         float* scale_out, double* avg_sigma_out);
 
+/* The server's record of its updates (Section 3.2: it "records the vector clock of each weight
+ * update to keep track of the average staleness"; Fig. 3 plots both).  rudra_ps_clock_log copies
+ * out, for the updates that advanced the timestamp from first_ts, first_ts + 1, ... (at most
+ * count of them, only the most recent 4096 are kept), the c gradient timestamps of each
+ * (pulled_ts_out, count * c entries, may be NULL) and its <sigma> by Eq. 2 (avg_sigma_out, count
+ * entries, may be NULL); returns how many were written, RUDRA_E_STATE if first_ts has left the
+ * log.  rudra_ps_staleness_histogram writes how many gradients had staleness 0, 1, ..., nbins - 1
+ * since create (set_weights and import_state do not reset it) and returns the number of bins
+ * needed to hold every value seen. */
+int64_t rudra_ps_clock_log(const rudra_ps* ps, uint64_t first_ts, uint64_t count, uint64_t* pulled_ts_out,
+                           double* avg_sigma_out);
+int64_t rudra_ps_staleness_histogram(const rudra_ps* ps, uint64_t* counts_out, uint32_t nbins);
+
 /* Checkpoint hooks: device-to-device copies of the weights and the state vector (either may be
  * NULL) out of / into the handle; import also sets the timestamp and empties the queue. */
 int rudra_ps_export_state(rudra_ps* ps, float* theta_dst_dev, float* state_dst_dev);

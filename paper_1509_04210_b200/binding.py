@@ -83,6 +83,8 @@ def lib():
         "rudra_sched_destroy": (None, [vp]),
         "rudra_sched_next": (i64, [vp, vp, u64]),
         "rudra_ps_run_events": (i64, [vp, vp, u64, vp, vp, u32]),
+        "rudra_ps_clock_log": (i64, [vp, u64, u64, vp, vp]),
+        "rudra_ps_staleness_histogram": (i64, [vp, vp, u32]),
         "rudra_ps_enable_views": (C.c_int, [vp, u32]),
         "rudra_ps_pull_view": (i64, [vp, u32, vp]),
         "rudra_ps_view_of": (i64, [vp, u32, vp]),
@@ -237,6 +239,19 @@ class ParameterServer:
         c = _check(lib().rudra_ps_last_clock(self._h, pulled.ctypes.data, sigma.ctypes.data, scale.ctypes.data,
                                              C.addressof(avg)))
         return {"c": c, "pulled_ts": pulled[:c], "sigma": sigma[:c], "scale": scale[:c], "avg_sigma": avg.value}
+
+    def clock_log(self, first_ts, count):
+        """(gradient timestamps [k, c], <sigma> [k]) of the updates first_ts, first_ts + 1, ..."""
+        pulled = np.zeros((count, self.c), dtype=np.uint64)
+        avg = np.zeros(count, dtype=np.float64)
+        k = _check(lib().rudra_ps_clock_log(self._h, int(first_ts), int(count), pulled.ctypes.data, avg.ctypes.data))
+        return pulled[:k], avg[:k]
+
+    def staleness_histogram(self):
+        need = _check(lib().rudra_ps_staleness_histogram(self._h, None, 0))
+        counts = np.zeros(max(need, 1), dtype=np.uint64)
+        _check(lib().rudra_ps_staleness_histogram(self._h, counts.ctypes.data, len(counts)))
+        return counts[:need]
 
     def export_state(self, theta_dst_dev=None, state_dst_dev=None):
         _check(lib().rudra_ps_export_state(self._h, _ptr(theta_dst_dev), _ptr(state_dst_dev)))

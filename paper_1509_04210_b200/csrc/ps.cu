@@ -2,6 +2,7 @@
 // (scalar timestamp, staleness, vector clock, Eq. 2), the step-size table of Eq. 5 / Eq. 6 and
 // the launches.  All floating-point work on the model happens in the kernels of update.cu and
 // snapshot.cu; nothing here touches a weight.
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdint>
@@ -90,6 +91,13 @@ struct rudra_ps {
   std::vector<uint32_t> sigma;
   std::vector<float> scale;
   double avg_sigma = 0.0;
+  // Record of past updates (Section 3.2: the server records the vector clock of each weight
+  // update to keep track of the average staleness): a ring of the last kClockLog updates, c
+  // gradient timestamps each, and a histogram of every staleness value seen since create.
+  static constexpr uint32_t kClockLog = 4096;
+  std::vector<uint64_t> log_pulled;     // kClockLog * c
+  std::vector<uint64_t> log_ts;         // timestamp before the update in that ring position, or ~0
+  std::vector<uint64_t> sigma_hist;     // count per staleness value, grown on demand
   uint64_t counters[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 
   // Zero-copy pulls (rudra_ps_enable_views): a pool of immutable weight versions.  A pull hands
@@ -238,6 +246,19 @@ void append_update(rudra_ps* ps, Window& w) {
     }
   }
   ps->avg_sigma = (double)ps->ts - (double)sum_pulled / (double)c;
+  {
+    if (ps->log_ts.empty()) {
+      ps->log_ts.assign(rudra_ps::kClockLog, ~0ull);
+      ps->log_pulled.assign((size_t)rudra_ps::kClockLog * c, 0);
+    }
+    const size_t pos = (size_t)(ps->ts % rudra_ps::kClockLog);
+    ps->log_ts[pos] = ps->ts;
+    for (uint32_t l = 0; l < c; ++l) {
+      ps->log_pulled[pos * c + l] = ps->clock[l];
+      if (ps->sigma[l] >= ps->sigma_hist.size()) ps->sigma_hist.resize((size_t)ps->sigma[l] + 1, 0);
+      ps->sigma_hist[ps->sigma[l]] += 1;
+    }
+  }
   double sum_scale = 0.0;
   for (uint32_t l = 0; l < c; ++l) {
     double divisor;
@@ -458,6 +479,7 @@ static int set_weights_common(rudra_ps* ps, const float* src, cudaMemcpyKind kin
   ps->ts = 0;
   ps->has_clock = false;
   for (auto& v : ps->versions) v.valid = false;   // held views keep their contents; none matches the new weights
+  std::fill(ps->log_ts.begin(), ps->log_ts.end(), ~0ull);   // timestamps start over: the log would be ambiguous
   return 0;
 }
 
@@ -765,6 +787,35 @@ int rudra_ps_last_clock(const rudra_ps* ps, uint64_t* pulled_ts_out, uint32_t* s
   return (int)ps->c;
 }
 
+int64_t rudra_ps_clock_log(const rudra_ps* ps, uint64_t first_ts, uint64_t count, uint64_t* pulled_ts_out,
+                           double* avg_sigma_out) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  uint64_t got = 0;
+  for (; got < count; ++got) {
+    const uint64_t t = first_ts + got;
+    if (t >= ps->ts || ps->log_ts.empty()) break;
+    const size_t pos = (size_t)(t % rudra_ps::kClockLog);
+    if (ps->log_ts[pos] != t) {
+      if (got == 0) return fail(RUDRA_E_STATE, "update %llu is no longer in the log (the last %u are kept)", (unsigned long long)t, rudra_ps::kClockLog);
+      break;
+    }
+    uint64_t sum = 0;
+    for (uint32_t l = 0; l < ps->c; ++l) {
+      const uint64_t p = ps->log_pulled[pos * ps->c + l];
+      if (pulled_ts_out) pulled_ts_out[got * ps->c + l] = p;
+      sum += p;
+    }
+    if (avg_sigma_out) avg_sigma_out[got] = (double)t - (double)sum / (double)ps->c;
+  }
+  return (int64_t)got;
+}
+
+int64_t rudra_ps_staleness_histogram(const rudra_ps* ps, uint64_t* counts_out, uint32_t nbins) {
+  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+  for (uint32_t b = 0; b < nbins && counts_out; ++b) counts_out[b] = b < ps->sigma_hist.size() ? ps->sigma_hist[b] : 0;
+  return (int64_t)ps->sigma_hist.size();
+}
+
 int rudra_ps_export_state(rudra_ps* ps, float* theta_dst_dev, float* state_dst_dev) {
   if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
   DeviceScope dev(ps->device);
@@ -788,6 +839,7 @@ int rudra_ps_import_state(rudra_ps* ps, const float* theta_src_dev, const float*
   ps->ts = ts;
   ps->has_clock = false;
   for (auto& v : ps->versions) v.valid = false;
+  std::fill(ps->log_ts.begin(), ps->log_ts.end(), ~0ull);
   return 0;
 }
 

@@ -273,3 +273,54 @@ def test_stress_config_full_size_backlog_sampled_against_oracle():
             assert torch.equal(slots[i], th)           # every learner received this version
     assert ps.counters()["launches"] == 6             # update + 128-way copy per window
     ps.close()
+
+
+def test_clock_log_and_staleness_histogram_match_the_trace():
+    """The server's record of its updates (vector clock per update, <sigma> of Eq. 2, staleness
+    histogram: the data behind the paper's Fig. 3) against the oracle and the event trace."""
+    from paper_1509_04210_b200 import binding as rb
+
+    lam, n, N = 30, 30, 2048                       # the lambda-softsync case of Section 5.1
+    w = synth.Workload("fig3b", N, lam, n, 0.001, 0.9, 0.0, synth.SOFTSYNC_ROUNDS, 0, 0.01, 1e-3)
+    rb_, th0, grads_np, grads, make = _setup(w, N)
+    ps, slots = make()
+    ev = rb.Scheduler(lam, n, w.mode, 3).next(9000)
+    pos = 0
+    while pos < len(ev):
+        ps.run_events(ev[pos:pos + 700], grads, slots)
+        pos += 700
+    ps.sync()
+    pushes = ev[ev["kind"] == rb.EV_PUSH]
+    K = ps.timestamp()
+    assert K == len(pushes) == 3000                # c = 1: every push is an update
+    pulled, avg = ps.clock_log(0, K)
+    assert len(avg) == K
+    np.testing.assert_array_equal(pulled[:, 0], pushes["pulled_ts"])
+    sigma = (pushes["ts"] - pushes["pulled_ts"]).astype(np.int64)
+    np.testing.assert_array_equal(avg, sigma.astype(np.float64))          # Eq. 2 with c = 1
+    hist = ps.staleness_histogram()
+    np.testing.assert_array_equal(hist, np.bincount(sigma, minlength=len(hist)))
+    assert abs(sigma[2 * lam:].mean() - 29.0) < 0.5 and sigma.max() <= 2 * n   # <sigma> close to 30, at most 2n
+    # a grouped case against the oracle's per-update records
+    w2 = synth.WORKLOADS["imagenet"]
+    rb_, th0, grads_np, grads, make = _setup(w2, 1024)
+    ps2, slots2 = make()
+    o = ora.OraclePS(1024, w2.lam, w2.n, w2.alpha0, w2.momentum, w2.weight_decay)
+    o.set_weights(th0)
+    ev = rb.Scheduler(w2.lam, w2.n, w2.mode, 3).next(2000)
+    ps2.run_events(ev, grads, slots2)
+    want_p, want_a = [], []
+    for e in ev:
+        if e["kind"] == ora.PUSH:
+            o.push(grads_np[int(e["learner"])], int(e["pulled_ts"]))
+        elif e["kind"] == ora.STEP:
+            o.step()
+            rec = o.last_clock()
+            want_p.append(rec["pulled_ts"].copy())
+            want_a.append(rec["avg_sigma"])
+    pulled, avg = ps2.clock_log(0, 10 ** 6)
+    np.testing.assert_array_equal(pulled, np.array(want_p))
+    np.testing.assert_array_equal(avg, np.array(want_a))
+    late, _ = ps2.clock_log(len(want_a) - 5, 100)
+    np.testing.assert_array_equal(late, np.array(want_p[-5:]))
+    ps.close(), ps2.close()
