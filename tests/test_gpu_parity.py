@@ -378,3 +378,28 @@ def test_queue_capacity_is_reported():
         done += 1
     assert done == rb.QUEUE_CAP // 128 and ps.timestamp() == done
     ps.close()
+
+
+def test_a_learner_that_never_pushes():
+    # n-softsync needs any c gradients (Eq. 5), so the server keeps advancing without learner 3;
+    # hardsync (c = lambda) waits, and the wait is a return value, never a device-side wait.
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    N = 4096
+    g = [to_device(synth.gradient(N, l, 0, 1e-2)) for l in range(4)]
+    soft = rb.ParameterServer(N, 4, 2, 0.1)            # c = 2
+    for k in range(9):
+        soft.push(g[k % 3], soft.timestamp())          # learners 0, 1, 2 only
+        assert soft.step() == (1 if k % 2 else 0)
+    assert soft.timestamp() == 4
+    hard = rb.ParameterServer(N, 4, 1, 0.1)            # c = 4
+    for l in range(3):
+        hard.push(g[l], 0)
+    for _ in range(5):
+        assert hard.step() == 0 and hard.timestamp() == 0
+    hard.sync()                                        # returns at once: nothing was launched
+    assert hard.counters()["launches"] == 0
+    hard.push(g[3], 0)
+    assert hard.step() == 1
+    soft.close(), hard.close()
