@@ -66,9 +66,18 @@ CASES = [
 ]
 
 
+EXTRA = {
+    # the widest group one launch can carry, with a 128-way broadcast after it
+    "hardsync128": synth.Workload("hardsync128", 3001, 128, 1, 0.01, 0.9, 5e-4, synth.HARDSYNC, 0, 0.01, 1e-2),
+    # 32 updates of 4 gradients fill the gradient table exactly
+    "fill_table": synth.Workload("fill_table", 5003, 128, 32, 0.01, 0.9, 5e-4, synth.SOFTSYNC_TIMED, 0, 0.01, 1e-2),
+}
+CASES += [("hardsync128", 3001, 800, 0), ("fill_table", 5003, 2500, 0), ("fill_table", 5003, 2500, 7)]
+
+
 @pytest.mark.parametrize("name,N,nevents,max_window", CASES)
 def test_backlog_equals_one_message_at_a_time(name, N, nevents, max_window):
-    w = synth.WORKLOADS[name]
+    w = synth.WORKLOADS.get(name) or EXTRA[name]
     rb, th0, grads_np, grads, make = _setup(w, N)
     ev = rb.Scheduler(w.lam, w.n, w.mode, 17, w.lognormal_sigma, w.downcast).next(nevents)
     a, slots_a = make()
