@@ -126,3 +126,16 @@ def test_workload_shapes():
     assert g.dtype == np.float32 and abs(float(g.std()) - 1e-3) < 2e-4
     np.testing.assert_array_equal(g, synth.gradient(1000, 3, 5, 1e-3))
     assert not np.array_equal(g, synth.gradient(1000, 3, 6, 1e-3))
+
+
+def test_bf16_rounding_recipe_agrees_with_torch():
+    # the input recipe rounds to nearest, ties to even; torch's cast is an independent implementation
+    import torch
+
+    rng = np.random.default_rng(0)
+    x = (rng.standard_normal(200000) * 1e-3).astype(np.float32)
+    ties = (np.arange(1, 2001, dtype=np.uint32) << np.uint32(16)) | np.uint32(0x8000)      # exactly halfway
+    x = np.concatenate([x, ties.view(np.float32), -ties.view(np.float32), np.float32([0.0, -0.0, 1.0, 65504.0])])
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(synth.to_bf16_bits(x), want)
+    np.testing.assert_array_equal(synth.bf16_bits_to_f32(want), torch.from_numpy(x).to(torch.bfloat16).float().numpy())
