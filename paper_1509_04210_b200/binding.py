@@ -165,7 +165,11 @@ class Scheduler:
             lib().rudra_sched_destroy(self._h)
             self._h = None
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:   # interpreter shutdown: the module may already be gone
+            pass
 
 
 class ParameterServer:
@@ -287,4 +291,8 @@ class ParameterServer:
             lib().rudra_ps_destroy(self._h)
             self._h = None
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:   # interpreter shutdown: the module may already be gone
+            pass

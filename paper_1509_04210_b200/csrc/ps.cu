@@ -179,6 +179,7 @@ int check_push(rudra_ps* ps, uint64_t pulled_ts) {
 // A launch under construction: a window of consecutive updates and the pulls between them.
 struct Window {
   rudra::UpdateParams p;
+  cudaError_t wait_error = cudaSuccess;   // first failure while ordering the launch after its uploads
   uint32_t nupd = 0, ndst = 0;
   uint32_t npulls = 0;           // learner pulls served (a shared version serves several with one copy)
   uint32_t nversions = 0;        // versions written by this launch
@@ -241,7 +242,8 @@ void append_update(rudra_ps* ps, Window& w) {
     sum_pulled += e.pulled_ts;
     p.grad[base + l] = e.grad;
     if (e.slot >= 0) {
-      cudaStreamWaitEvent(ps->stream, ps->slot_ready[e.slot], 0);   // the kernel starts after its uploads
+      const cudaError_t we = cudaStreamWaitEvent(ps->stream, ps->slot_ready[e.slot], 0);   // the kernel starts after its uploads
+      if (we != cudaSuccess && w.wait_error == cudaSuccess) w.wait_error = we;
       w.used_slots.push_back(e.slot);
     }
   }
@@ -293,7 +295,8 @@ int flush_window(rudra_ps* ps, Window& w) {
     w.npulls = 0;
     return 0;
   }
-  cudaError_t e = cudaSuccess;
+  cudaError_t e = w.wait_error;
+  w.wait_error = cudaSuccess;
   uint32_t launches = 0;
   auto copy_weights = [&](uint32_t d0, uint32_t d1) {   // 1 -> (d1 - d0) copy of the current weights
     if (d1 == d0 || e != cudaSuccess) return;
@@ -338,7 +341,8 @@ int flush_window(rudra_ps* ps, Window& w) {
     if (split) copy_weights(pre, post);
   }
   for (int slot : w.used_slots) {   // the next upload into the slot waits for this launch
-    cudaEventRecord(ps->slot_spent[slot], ps->stream);
+    const cudaError_t re = cudaEventRecord(ps->slot_spent[slot], ps->stream);
+    if (re != cudaSuccess && e == cudaSuccess) e = re;
     ps->free_slots.push_back(slot);
   }
   ps->counters[1] += w.nupd;
@@ -509,7 +513,11 @@ int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_
   if (!ps->free_slots.empty()) {
     slot = ps->free_slots.back();
     ps->free_slots.pop_back();
-    cudaStreamWaitEvent(ps->up_stream, ps->slot_spent[slot], 0);   // its last reader must be done
+    e = cudaStreamWaitEvent(ps->up_stream, ps->slot_spent[slot], 0);   // its last reader must be done
+    if (e != cudaSuccess) {
+      ps->free_slots.push_back(slot);
+      return cuda_fail(e, "cudaStreamWaitEvent");
+    }
   } else {
     void* buf = nullptr;
     cudaEvent_t ready = nullptr, spent = nullptr;
@@ -749,7 +757,8 @@ int64_t rudra_ps_pull_host(rudra_ps* ps, float* dst_host) {
   rudra_ps::DownBuf& d = ps->down[ps->down_next++ % ps->down.size()];
   // snapshot on the main stream (after every update issued so far), then the copy to the host
   // on the download stream, so later updates need not wait for PCIe
-  cudaStreamWaitEvent(ps->stream, d.drained, 0);
+  e = cudaStreamWaitEvent(ps->stream, d.drained, 0);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent");
   rudra::SnapshotParams sp;
   sp.dst[0] = d.buf;
   sp.src = ps->theta;
