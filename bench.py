@@ -223,6 +223,33 @@ def oracle_run(w, windows, nsample, grads_host, warmup=0, budget_s=None, max_win
     return done, time.perf_counter() - t0
 
 
+def oracle_run_all_cores(w, windows, grads_host, cores, budget_s, adagrad=False):
+    """The same oracle, one unmodified single-threaded instance per core on disjoint slices of the
+    vector (the path is element-wise, so slicing changes nothing); returns (windows done, seconds)."""
+    import threading as th
+
+    n = len(grads_host[0])
+    bounds = [n * i // cores for i in range(cores + 1)]
+    results = [None] * cores
+    # fix the number of windows from a short probe so that all threads do the same work
+    probe_done, probe_dt = oracle_run(w, windows, min(n, 1 << 20), [g[: 1 << 20] for g in grads_host], warmup=0,
+                                      max_windows=2, adagrad=adagrad)
+    per_window = probe_dt / probe_done * (n / cores) / min(n, 1 << 20)
+    todo = max(2, min(len(windows), int(budget_s / max(per_window, 1e-9))))
+
+    def work(i):
+        sl = [np.ascontiguousarray(g[bounds[i]: bounds[i + 1]]) for g in grads_host]
+        results[i] = oracle_run(w, windows, bounds[i + 1] - bounds[i], sl, warmup=0, max_windows=todo, adagrad=adagrad)
+
+    threads = [th.Thread(target=work, args=(i,)) for i in range(cores)]
+    t0 = time.perf_counter()
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    return todo, time.perf_counter() - t0
+
+
 def host_gradients(w, nsample, count):
     return [synth.gradient(nsample, l, 0, w.grad_std, w.grad_dtype) for l in range(count)]
 
@@ -518,6 +545,15 @@ def run_ours(args, w):
                           % (done, nh, dt),
                 "host_cores_available": os.cpu_count(),
             }
+            cores = os.cpu_count() or 1
+            if cores > 1:
+                done_all, dt_all = oracle_run_all_cores(w, windows, grads, cores, 8.0, adagrad=args.optimizer == "adagrad")
+                line["cpu_baseline"]["all_cores"] = {
+                    "value": done_all / dt_all, "unit": UNIT, "cores": cores,
+                    "kind": "oracle, one unmodified single-threaded instance per core on disjoint slices of the vector",
+                    "sample": "%d full-size update windows, %.1f s (slicing and per-thread copies of the inputs included)"
+                              % (done_all, dt_all),
+                }
         print(json.dumps(line), flush=True)
     ps.close()
     if world > 1:
