@@ -421,6 +421,31 @@ def run_ours(args, w):
     pulls = c1["pulls"] - c0["pulls"]
     copies = c1["weight_copies"] - c0["weight_copies"]
 
+    # What HBM delivers on this GPU, in this run, for the same mix of reads and writes as one launch
+    # of the dominant kernel: a probe kernel that only streams that many vectors in and out.
+    mix = None
+    if W >= 1 and not views and w.grad_dtype == synth.GRAD_F32 and N * 8 > 126e6 and nbufs == w.lam:
+        per_launch = max(1, args.steps // max(len(timed), 1))
+        nr = min(64, per_launch * w.c + state_bytes(w) // 8)
+        nw = min(64, int(round(copies / max(len(timed), 1))) + state_bytes(w) // 8)
+        extra = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(4)]
+        srcs = (bufs + extra[:2])[-nr:] if nr <= len(bufs) + 2 else None
+        dsts = (slots + extra[2:])[-nw:] if nw <= len(slots) + 2 else None
+        if srcs and dsts:
+            for _ in range(3):
+                rb.stream_probe(srcs, dsts, N, stream)
+            p0, p1 = new_events()
+            reps = 10
+            p0.record(stream)
+            for _ in range(reps):
+                rb.stream_probe(srcs, dsts, N, stream)
+            p1.record(stream)
+            torch.cuda.synchronize()
+            mix = {"gbs": 4.0 * N * (nr + nw) * reps / (p0.elapsed_time(p1) * 1e-3) / 1e9, "reads": nr, "writes": nw,
+                   "launches": reps,
+                   "how": "rudra_stream_probe: the same number of vectors streamed in and out, same access shape, no arithmetic"}
+        del extra
+
     e2e_ms, e2e_steps, h0, h1 = float('nan'), 0, None, None
     if not args.kernel_only:
         # end to end through the C interface with host buffers: gradients travel host -> device inside
@@ -528,6 +553,8 @@ def run_ours(args, w):
                     "last_tenth": 1e3 * float(np.mean(launch_ms[-max(1, len(launch_ms) // 10):]))},
                 "frac_of_8TBs_datasheet": achieved / 8000.0,
                 "traffic": ncu_traffic(w.name, W, N),
+                "mix_ceiling": mix,
+                "frac_of_mix_ceiling": None if not mix else achieved / mix["gbs"],
             },
         }
         if world == 1 and not args.no_cpu_baseline and not args.kernel_only:

@@ -241,6 +241,17 @@ int rudra_ps_update_host_noalloc(float* theta_dev, float* state_dev, uint64_t np
                                  float momentum, float weight_decay, void* cuda_stream);
 const char* rudra_noalloc_last_error(void);
 
+/*
+ * rudra_stream_probe -- measurement utility; the paper has no counterpart.  Enqueues one kernel
+ * that reads nreads vectors (srcs_dev) and writes nwrites vectors (dsts_dev; their contents become
+ * meaningless), nfloats floats each, 32-byte aligned, at most 64 of each, with the update
+ * kernel's access shape and nothing else.  Timing it gives the bandwidth this GPU sustains for
+ * that mix of reads and writes, the ceiling against which the update kernel's own figure is to be
+ * read.  Returns 0, RUDRA_E_INVAL or RUDRA_E_CUDA.
+ */
+int rudra_stream_probe(const float* const* srcs_dev, uint32_t nreads, float* const* dsts_dev,
+                       uint32_t nwrites, uint64_t nfloats, void* cuda_stream);
+
 /* ------------------------------------------------------------------------------------------
  * Learner event model.  The paper's server handles incoming messages strictly one by one
  * (Section 3.2), which makes the arrival order the whole control; this host-only scheduler

@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_PKG, "librudra_ps.so")
-SOURCES = ["ps.cu", "update.cu", "snapshot.cu", "noalloc.cu", "sched.cpp"]
+SOURCES = ["ps.cu", "update.cu", "snapshot.cu", "noalloc.cu", "probe.cu", "sched.cpp"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-cudart", "static", "-shared",
