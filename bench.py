@@ -587,6 +587,34 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_probe_mixes(args, w):
+    """--probe-mixes: what HBM delivers for mixes of reads and writes (rudra_stream_probe), as a table."""
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    N = w.nparams
+    pool = [torch.zeros(N, dtype=torch.float32, device="cuda") for _ in range(120)]
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    print("vector length %d floats, distinct vectors rotating through a pool of %d, 8 timed launches each" % (N, len(pool)))
+    for nr, nw in [(54, 0), (0, 54), (27, 27), (56, 56), (20, 8), (56, 2), (2, 56), (40, 16), (16, 40), (8, 0), (0, 8)]:
+        def launch(i):
+            srcs = [pool[(i * 7 + l) % 60] for l in range(nr)]
+            dsts = [pool[60 + (i * 5 + l) % 60] for l in range(nw)]
+            rb.stream_probe(srcs, dsts, N, stream)
+        for i in range(2):
+            launch(i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(8):
+            launch(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / 8 * 1e3
+        print("reads %2d writes %2d  write share %.2f  %8.1f us  %6.0f GB/s"
+              % (nr, nw, nw / (nr + nw), us, 4.0 * N * (nr + nw) / us * 1e-3), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -602,6 +630,8 @@ def main():
                     help="copy: every pull writes the learner's own slot; views: zero-copy shared weight versions")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adagrad"],
                     help="momentum SGD with weight decay (Section 4.2) or AdaGrad at the server (Section 5.5)")
+    ap.add_argument("--probe-mixes", action="store_true",
+                    help="print what HBM delivers for several mixes of reads and writes (no bench line) and exit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-only", action="store_true",
                     help="device-resident timed region only: no end-to-end leg, no CPU baseline (profiler captures)")
@@ -628,6 +658,9 @@ def main():
         import dataclasses
 
         w = dataclasses.replace(w, name=w.name + "@%d" % args.nparams, nparams=args.nparams)
+    if args.probe_mixes:
+        run_probe_mixes(args, w)
+        return
     if args.impl == "reference":
         run_reference(args, w)
     else:
