@@ -341,7 +341,10 @@ def run_ours(args, w):
         ps.enable_views(w.lam + 1)
     ps.sync()
     ps.set_stream(stream)
-    windows = make_windows(w, args.warmup + args.steps)
+    extra_steps = 0 if (args.window == 0 or args.pull == "views") else min(args.steps, 216)
+    windows = make_windows(w, args.warmup + args.steps + extra_steps)
+    extra_windows = windows[args.warmup + args.steps:]
+    windows = windows[: args.warmup + args.steps]
     W = default_window(w, views) if args.window < 0 else args.window
     if views and W == 0:
         raise SystemExit("--pull views is served through rudra_ps_run_events: use --window >= 1")
@@ -420,6 +423,25 @@ def run_ours(args, w):
     launches = c1["launches"] - c0["launches"]
     pulls = c1["pulls"] - c0["pulls"]
     copies = c1["weight_copies"] - c0["weight_copies"]
+
+    # The same server, continuing the same event stream, driven one message at a time (push, step,
+    # pull as separate calls and launches): the unbatched figure beside the backlog figure.
+    single = None
+    if extra_steps and W != 0:
+        fill_event_pool(extra_steps + 2)
+        sev = []
+        barrier()
+        s0, s1 = new_events()
+        s0.record(stream)
+        for win in extra_windows:
+            run_messages(win, sev)
+        s1.record(stream)
+        barrier()
+        sms = replicas.max_over_ranks([s0.elapsed_time(s1)], device="cuda")[0]
+        upd_us = 1e3 * float(np.mean([a.elapsed_time(b) for a, b in sev]))
+        single = {"value": replicas.whole_job_rate(extra_steps, world, sms), "unit": UNIT, "steps": extra_steps,
+                  "update_kernel_us": upd_us,
+                  "update_kernel_gbs": update_bytes_per_param(w) * N / (upd_us * 1e-6) / 1e9}
 
     # What HBM delivers on this GPU, in this run, for the same mix of reads and writes as one launch
     # of the dominant kernel: a probe kernel that only streams that many vectors in and out.
@@ -533,6 +555,7 @@ def run_ours(args, w):
             "bytes_per_param_per_step": path_bytes / N / args.steps,
             "pulls_per_step": pulls / args.steps,
             "weight_copies_per_step": copies / args.steps,
+            "one_message_at_a_time": single,
             "gpu_launches": launches,
             "clocks": clocks,
             "e2e": None if args.kernel_only else {
