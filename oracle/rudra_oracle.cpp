@@ -19,7 +19,10 @@
 //   * sigma = 0 floor in the per-gradient and group-mean rate policies
 //     (alpha0/sigma is undefined at sigma = 0)  : parity unpinned by the paper.
 //   * AdaGrad form (Section 5.5 names the method, prints no formula)
-//                                           : parity unpinned by the paper.
+//                                           : parity unpinned by the paper; the
+//     reading at OraclePS::step is pinned by the direction of the first step
+//     (the sign of gradient plus penalty), by a decay-only scalar recurrence
+//     and by brute force in decimal arithmetic with unequal per-gradient rates.
 // Everything else is pinned by Eq. 2-6 and the staleness sets printed in
 // Section 5.1 (see tests/).
 //

@@ -307,6 +307,131 @@ def test_adagrad_constant_gradient_closed_form():
     _close(ps.state(), K * g64 * g64, 0.0, ulps=2.0 * K)
 
 
+def _adagrad_reference(th0, grads_per_step, weights_per_step, abar_per_step, wd, eps, digits=60):
+    """Reading of AdaGrad at the server carried out in 60-digit decimal arithmetic, one weight at a
+    time: gbar = sum_l w_l g_l + wd theta;  h += gbar^2;  theta -= abar gbar / (sqrt(h) + eps)."""
+    from decimal import Decimal, getcontext
+
+    getcontext().prec = digits
+    D = lambda x: Decimal(float(x))
+    th = [D(x) for x in th0]
+    h = [Decimal(0)] * len(th)
+    for grads, weights, abar in zip(grads_per_step, weights_per_step, abar_per_step):
+        for k in range(len(th)):
+            gbar = sum((Decimal(w) * D(g[k]) for w, g in zip(weights, grads)), Decimal(0)) + D(wd) * th[k]
+            h[k] = h[k] + gbar * gbar
+            th[k] = th[k] - Decimal(abar) * gbar / (h[k].sqrt() + D(eps))
+    return np.array([float(x) for x in th]), np.array([float(x) for x in h])
+
+
+def test_adagrad_decay_only_follows_the_scalar_recurrence():
+    # g = 0, wd > 0: the only force is the L2 penalty, gbar = wd theta.  The first step is then
+    # theta_1 = theta_0 - abar theta_0 / (|theta_0| + eps / wd): every weight moves towards zero by (almost
+    # exactly) abar whatever its size; later steps follow the scalar recurrence, evaluated in decimal.
+    N, K, a0, wd = 12, 7, 0.003, 0.25
+    ps, th0 = _mk(N, 4, 2, a0, wd=wd)
+    ps.set_optimizer(ora.OPT_ADAGRAD, 1e-8)
+    z = np.zeros(N, dtype=np.float32)
+    abar = float(np.float32(2 * float(np.float32(float(np.float32(a0)) / 4.0))))
+    ps.push(z, 0), ps.push(z, 0)
+    assert ps.step() == 1
+    th1 = ps.pull()[0].astype(np.float64)
+    np.testing.assert_allclose(th0 - th1, abar * np.sign(th0), rtol=1e-4)      # moved by abar towards zero
+    for _ in range(K - 1):
+        ps.push(z, ps.timestamp()), ps.push(z, ps.timestamp())
+        assert ps.step() == 1
+    want_th, want_h = _adagrad_reference(th0, [[z, z]] * K, [["0.5", "0.5"]] * K, [repr(abar)] * K,
+                                         np.float32(wd), np.float32(1e-8))
+    _close(ps.pull()[0], want_th, 1e-3, ulps=4.0 * K)
+    _close(ps.state(), want_h, 0.0, ulps=4.0 * K)
+    assert np.all(want_h > 0)            # a dropped penalty term would leave h = 0 and theta unmoved
+
+
+def test_adagrad_first_step_direction_is_the_sign_of_gradient_plus_decay():
+    # From h = 0 the first AdaGrad step is abar gbar / (|gbar| + eps) = abar sign(gbar): its direction
+    # reveals gbar's sign.  theta = 1, g = -0.05, wd = 0.1, abar = 0.1: g + wd theta = +0.05 (weight falls);
+    # without the penalty, or with the penalty taken at abar wd, gbar would be negative (weight rises).
+    N = 4
+    a0, wd = 0.1, 0.1
+    ps = ora.OraclePS(N, 1, 1, a0, 0.0, wd)
+    ps.set_optimizer(ora.OPT_ADAGRAD, 1e-8)
+    ps.set_weights(np.array([1.0, -1.0, 1.0, -1.0], dtype=np.float32))
+    ps.push(np.array([-0.05, 0.05, -0.2, 0.2], dtype=np.float32), 0)
+    assert ps.step() == 1
+    got = ps.pull()[0].astype(np.float64)
+    a = float(np.float32(a0))
+    # weights 0, 1: the penalty wins (+0.05 / -0.05); weights 2, 3: the gradient wins (-0.1 / +0.1)
+    np.testing.assert_allclose(got, [1.0 - a, -1.0 + a, 1.0 + a, -1.0 - a], rtol=1e-6)
+
+
+def test_adagrad_per_gradient_weights_are_step_sizes_over_their_sum():
+    # c = 3 under the per-gradient policy with staleness (0, 4, 1): divisors (1, 4, 1), step sizes
+    # a/3, a/12, a/3, their sum abar = 3a/4, weights s_l / abar = 4/9, 1/9, 4/9.
+    # Direction pin: g = (1, -3, 1) x has weighted mean +5x/9 but plain mean -x/3, so the first step
+    # (abar sign(gbar)) goes opposite ways under the two weightings.
+    N, a0 = 6, 0.12
+    ps, _ = _mk(N, 6, 2, a0)
+    ps.set_policy(ora.LR_PER_GRADIENT)
+    _advance(ps, N, 6)                                   # plain SGD on zero gradients: weights unchanged, ts = 6
+    ps.set_optimizer(ora.OPT_ADAGRAD, 1e-8)
+    th = ps.pull()[0].astype(np.float64)
+    x = np.float32(0.01) * np.array([1, -1, 2, -2, 3, -3], dtype=np.float32)
+    gs = [x, np.float32(-3) * x, x]
+    for g, p in zip(gs, (6, 2, 5)):
+        ps.push(g, p)
+    assert ps.step() == 1
+    rec = ps.last_clock()
+    assert list(rec["sigma"]) == [0, 4, 1]
+    a = float(np.float32(a0))
+    assert rec["abar"] == pytest.approx(0.75 * a, rel=1e-6)
+    got = ps.pull()[0].astype(np.float64)
+    np.testing.assert_allclose(th - got, 0.75 * a * np.sign(x), rtol=1e-5)
+    # Second step on the same group (now stale by 1, 5, 2 -> divisors 1, 5, 2): sizes matter too.
+    for g, p in zip(gs, (6, 2, 5)):
+        ps.push(g, p)
+    assert ps.step() == 1
+    assert list(ps.last_clock()["sigma"]) == [1, 5, 2]
+    s2 = [float(np.float32(a / (d * 3))) for d in (1, 5, 2)]
+    abar2 = float(np.float32(sum(s2)))
+    want_th, want_h = _adagrad_reference(
+        th, [gs, gs], [["0.4444444444444444444444", "0.1111111111111111111111", "0.4444444444444444444444"],
+                       [repr(s / abar2) for s in s2]],
+        [repr(float(np.float32(sum(float(np.float32(a / (d * 3))) for d in (1, 4, 1))))), repr(abar2)], 0.0, np.float32(1e-8))
+    _close(ps.pull()[0], want_th, 1e-3, ulps=16.0)
+    _close(ps.state(), want_h, 0.0, ulps=16.0)
+    assert abs(abar2 / a - (1 / 3 + 1 / 15 + 1 / 6)) < 1e-6
+
+
+def test_adagrad_brute_force_on_a_tiny_vector():
+    # Everything at once on 5 weights: three gradients per update with unequal staleness, weight
+    # decay, changing rates; decimal arithmetic, divisors and weights worked out here from the
+    # staleness the test itself imposes.
+    N, a0, wd, K = 5, 0.09, 0.05, 6
+    ps, _ = _mk(N, 6, 2, a0, wd=wd, seed=11)
+    ps.set_policy(ora.LR_PER_GRADIENT)
+    ps.set_optimizer(ora.OPT_ADAGRAD, 1e-8)
+    th0 = ps.pull()[0].astype(np.float64)
+    a = float(np.float32(a0))
+    grads, weights, abars = [], [], []
+    for k in range(K):
+        ts = ps.timestamp()
+        lags = [min(ts, d) for d in (0, k, 2)]            # staleness imposed on the three gradients
+        gs = [synth.gradient(N, l, k, 1e-2, seed=11) for l in range(3)]
+        for g, lag in zip(gs, lags):
+            ps.push(g, ts - lag)
+        assert ps.step() == 1
+        s = [float(np.float32(a / (max(lag, 1) * 3))) for lag in lags]
+        abar = float(np.float32(sum(s)))
+        grads.append(gs), weights.append([repr(x / abar) for x in s]), abars.append(repr(abar))
+        assert list(ps.last_clock()["sigma"]) == lags
+    want_th, want_h = _adagrad_reference(th0, grads, weights, abars, np.float32(wd), np.float32(1e-8))
+    _close(ps.pull()[0], want_th, 1e-3, ulps=4.0 * K)
+    _close(ps.state(), want_h, 1e-9, ulps=4.0 * K)
+    # the penalty is visible at this size: the same run without it ends elsewhere
+    no_wd, _ = _adagrad_reference(th0, grads, weights, abars, 0.0, np.float32(1e-8))
+    assert np.abs(no_wd - want_th).max() > 50 * F32_EPS * np.abs(want_th).max()
+
+
 def test_strict_fp32_mode_tracks_the_double_mode():
     # the fp32 evaluation is the same rule: after a few updates it differs only by fp32 rounding
     N, lam, n = 500, 6, 2
