@@ -307,6 +307,7 @@ def run_ours(args, w):
     import torch
     import torch.distributed as dist
     from paper_1509_04210_b200 import binding as rb
+    from paper_1509_04210_b200 import probe
 
     from paper_1509_04210_b200 import replicas
 
@@ -455,12 +456,12 @@ def run_ours(args, w):
         dsts = (slots + extra[2:])[-nw:] if nw <= len(slots) + 2 else None
         if srcs and dsts:
             for _ in range(3):
-                rb.stream_probe(srcs, dsts, N, stream)
+                probe.stream_probe(srcs, dsts, N, stream)
             p0, p1 = new_events()
             reps = 10
             p0.record(stream)
             for _ in range(reps):
-                rb.stream_probe(srcs, dsts, N, stream)
+                probe.stream_probe(srcs, dsts, N, stream)
             p1.record(stream)
             torch.cuda.synchronize()
             mix = {"gbs": 4.0 * N * (nr + nw) * reps / (p0.elapsed_time(p1) * 1e-3) / 1e9, "reads": nr, "writes": nw,
@@ -613,7 +614,7 @@ def run_ours(args, w):
 def run_probe_mixes(args, w):
     """--probe-mixes: what HBM delivers for mixes of reads and writes (rudra_stream_probe), as a table."""
     import torch
-    from paper_1509_04210_b200 import binding as rb
+    from paper_1509_04210_b200 import probe
 
     N = w.nparams
     pool = [torch.zeros(N, dtype=torch.float32, device="cuda") for _ in range(120)]
@@ -624,7 +625,7 @@ def run_probe_mixes(args, w):
         def launch(i):
             srcs = [pool[(i * 7 + l) % 60] for l in range(nr)]
             dsts = [pool[60 + (i * 5 + l) % 60] for l in range(nw)]
-            rb.stream_probe(srcs, dsts, N, stream)
+            probe.stream_probe(srcs, dsts, N, stream)
         for i in range(2):
             launch(i)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -47,10 +47,12 @@ typedef struct rudra_sched rudra_sched;
 #define RUDRA_E_QUEUE_FULL (-3) /* more than RUDRA_QUEUE_CAP gradients waiting                   */
 #define RUDRA_E_CUDA       (-4) /* a CUDA call failed; text in rudra_last_error()                */
 #define RUDRA_E_STATE      (-5) /* call not legal in the current state (e.g. queue not empty)    */
+#define RUDRA_E_NOMEM      (-6) /* host memory ran out inside the call; destroy the handle       */
 
 #define RUDRA_MAX_GROUP  128    /* largest c = floor(lambda / n) one update can combine          */
 #define RUDRA_MAX_DSTS   128    /* most destinations of one pull_many / step_pull_many           */
 #define RUDRA_QUEUE_CAP  4096   /* most gradients that may wait in the queue                     */
+#define RUDRA_HIST_BINS  4096   /* staleness histogram: the last bin counts this much and more   */
 
 /* rudra_ps_set_option keys and values */
 #define RUDRA_OPT_GRAD_DTYPE 1
@@ -152,15 +154,17 @@ int64_t rudra_ps_timestamp(const rudra_ps* ps);
 int rudra_ps_last_clock(const rudra_ps* ps, uint64_t* pulled_ts_out, uint32_t* sigma_out,
                         float* scale_out, double* avg_sigma_out);
 
-/* The server's record of its updates (Section 3.2: it "records the vector clock of each weight
- * update to keep track of the average staleness"; Fig. 3 plots both).  rudra_ps_clock_log copies
+/* The server's record of its updates: Section 3.2 has the server log every update's vector clock
+ * so that the average staleness can be followed over training (Fig. 3 plots both).
+ * rudra_ps_clock_log copies
  * out, for the updates that advanced the timestamp from first_ts, first_ts + 1, ... (at most
  * count of them, only the most recent 4096 are kept), the c gradient timestamps of each
  * (pulled_ts_out, count * c entries, may be NULL) and its <sigma> by Eq. 2 (avg_sigma_out, count
  * entries, may be NULL); returns how many were written, RUDRA_E_STATE if first_ts has left the
  * log.  rudra_ps_staleness_histogram writes how many gradients had staleness 0, 1, ..., nbins - 1
  * since create (set_weights and import_state do not reset it) and returns the number of bins
- * needed to hold every value seen. */
+ * needed to hold every value seen, at most RUDRA_HIST_BINS: the bin RUDRA_HIST_BINS - 1 also counts
+ * every larger staleness. */
 int64_t rudra_ps_clock_log(const rudra_ps* ps, uint64_t first_ts, uint64_t count, uint64_t* pulled_ts_out,
                            double* avg_sigma_out);
 int64_t rudra_ps_staleness_histogram(const rudra_ps* ps, uint64_t* counts_out, uint32_t nbins);
@@ -181,8 +185,8 @@ int rudra_ps_counters(const rudra_ps* ps, uint64_t out[8]);
 
 /*
  * Zero-copy pulls.  Section 3.3 gives each learner a computation buffer and a communication
- * buffer for pullWeights, so that using newly received weights "only requires a pointer swap".
- * With learners and server sharing one GPU's memory the same idea removes the copy: the handle
+ * buffer for pullWeights, so that switching to newly received weights costs an exchange of two
+ * pointers and no copy.  With learners and server sharing one GPU's memory the same idea removes the copy: the handle
  * keeps a pool of nversions immutable weight vectors, a pull hands the learner a pointer to the
  * one holding the current timestamp, and learners that pull the same timestamp share it -- a
  * version is written once (4 bytes per weight, by the update kernel when the pull sits in a
@@ -232,25 +236,21 @@ const char* rudra_last_error(void);
  * one stream do not.  The array keeps the last call's gradients; nothing in it needs clearing
  * because each call overwrites all it reads.  The first call on each device looks up the array's
  * device address (cudaGetSymbolAddress, with that device current); make that first call before
- * any stream capture begins.  Returns 0, or RUDRA_E_INVAL / RUDRA_E_CUDA with the reason in
- * rudra_noalloc_last_error().
+ * any stream capture begins.  That first call is also where the CUDA runtime may load the
+ * library's device image onto the device, which is when the 16 MiB become resident: a process
+ * that is about to hand the rest of the GPU to its own pool should make one call (any small
+ * update) on each device before it does so.
+ * Host buffers: the gradients are copied with cudaMemcpyAsync.  From pageable memory the copy has
+ * left grads_host[l] when the call returns; from page-locked memory it is asynchronous, and
+ * grads_host[l] must stay unchanged until cuda_stream has passed the copies (an event recorded on
+ * cuda_stream after the call, or a synchronise).  scales is read before the call returns.
+ * Returns 0, or RUDRA_E_INVAL / RUDRA_E_CUDA with the reason in rudra_noalloc_last_error().
  */
 #define RUDRA_NOALLOC_MAX_FLOATS (4u * 1024u * 1024u)
 int rudra_ps_update_host_noalloc(float* theta_dev, float* state_dev, uint64_t nparams,
                                  const float* const* grads_host, const float* scales, uint32_t c,
                                  float momentum, float weight_decay, void* cuda_stream);
 const char* rudra_noalloc_last_error(void);
-
-/*
- * rudra_stream_probe -- measurement utility; the paper has no counterpart.  Enqueues one kernel
- * that reads nreads vectors (srcs_dev) and writes nwrites vectors (dsts_dev; their contents become
- * meaningless), nfloats floats each, 32-byte aligned, at most 64 of each, with the update
- * kernel's access shape and nothing else.  Timing it gives the bandwidth this GPU sustains for
- * that mix of reads and writes, the ceiling against which the update kernel's own figure is to be
- * read.  Returns 0, RUDRA_E_INVAL or RUDRA_E_CUDA.
- */
-int rudra_stream_probe(const float* const* srcs_dev, uint32_t nreads, float* const* dsts_dev,
-                       uint32_t nwrites, uint64_t nfloats, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
  * Learner event model.  The paper's server handles incoming messages strictly one by one
@@ -304,8 +304,11 @@ int64_t rudra_sched_next(rudra_sched* s, rudra_event* out, uint64_t count);
  * rudra_ps_push), slots_dev[l] its weight buffer (written by its pulls and by broadcasts); both
  * are host arrays of lambda device pointers; slots_dev may be NULL if no event pulls.  The events'
  * ts fields are checked against the server's timestamp.  The whole batch is validated before
- * anything is queued or launched: on a negative return nothing has changed.  Returns the number
- * of updates performed.
+ * anything is queued or launched: RUDRA_E_INVAL, RUDRA_E_BAD_TS, RUDRA_E_STATE and
+ * RUDRA_E_QUEUE_FULL mean that nothing has changed.  RUDRA_E_CUDA (a launch the driver refused) or
+ * RUDRA_E_NOMEM can come after part of the batch was handled: timestamp, queue and counters then
+ * stand where the failure left them, the weights may hold some of the batch's updates, and the
+ * handle is only good for rudra_ps_destroy.  Returns the number of updates performed.
  */
 int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t count,
                             const void* const* grads_dev, float* const* slots_dev, uint32_t max_window);

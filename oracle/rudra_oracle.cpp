@@ -295,9 +295,10 @@ struct OraclePS {
       } else {
         // AdaGrad at the server (Section 5.5), reading: the averaged gradient of Eq. 5 plus the
         // L2 penalty feeds a running sum of squares; the step is rate * g / (sqrt(sum) + eps).
+        // (with a zero rate every step size is 0: the weights are then Eq. 5's plain 1/c)
         double gbar = 0.0;
         for (uint32_t l = 0; l < c; ++l)
-          gbar += ((double)scale[l] / (double)abar) * grad_at(grp[l].grad, k);
+          gbar += (abar > 0.f ? (double)scale[l] / (double)abar : 1.0 / (double)c) * grad_at(grp[l].grad, k);
         gbar += (double)wd * (double)theta[k];
         double h = (double)vel[k] + gbar * gbar;
         double th = (double)theta[k] - (double)abar * gbar / (std::sqrt(h) + (double)adagrad_eps);
@@ -324,7 +325,7 @@ struct OraclePS {
         vel[k] = v;
       } else {
         for (uint32_t l = 0; l < c; ++l) {
-          const float wl = (float)((double)scale[l] / (double)abar);
+          const float wl = abar > 0.f ? (float)((double)scale[l] / (double)abar) : (float)(1.0 / (double)c);
           acc = std::fmaf(wl, (float)grad_at(grp[l].grad, k), acc);
         }
         const float g = std::fmaf(wd, theta[k], acc);

@@ -14,8 +14,8 @@ import numpy as np
 from . import build as _build
 
 # constants of include/rudra_ps.h
-E_INVAL, E_BAD_TS, E_QUEUE_FULL, E_CUDA, E_STATE = -1, -2, -3, -4, -5
-MAX_GROUP, MAX_DSTS, QUEUE_CAP = 128, 128, 4096
+E_INVAL, E_BAD_TS, E_QUEUE_FULL, E_CUDA, E_STATE, E_NOMEM = -1, -2, -3, -4, -5, -6
+MAX_GROUP, MAX_DSTS, QUEUE_CAP, HIST_BINS = 128, 128, 4096, 4096
 OPT_GRAD_DTYPE, OPT_LR_POLICY, OPT_OPTIMIZER = 1, 2, 3
 GRAD_F32, GRAD_BF16 = 0, 1
 LR_PAPER_N, LR_PER_GRADIENT, LR_GROUP_MEAN = 0, 1, 2
@@ -79,7 +79,6 @@ def lib():
         "rudra_last_error": (C.c_char_p, []),
         "rudra_ps_update_host_noalloc": (C.c_int, [vp, vp, u64, vp, vp, u32, f32, f32, vp]),
         "rudra_noalloc_last_error": (C.c_char_p, []),
-        "rudra_stream_probe": (C.c_int, [vp, u32, vp, u32, u64, vp]),
         "rudra_sched_create": (vp, [u32, u32, C.c_int, u64, C.c_double, C.c_int]),
         "rudra_sched_destroy": (None, [vp]),
         "rudra_sched_next": (i64, [vp, vp, u64]),
@@ -145,16 +144,6 @@ def update_host_noalloc(theta_dev, state_dev, nparams, grads_host, scales, momen
                                               momentum, weight_decay, handle)
     if code < 0:
         raise RudraError(code, lib().rudra_noalloc_last_error().decode())
-    return code
-
-
-def stream_probe(srcs_dev, dsts_dev, nfloats, stream=None):
-    """rudra_stream_probe: one launch that only reads srcs_dev and writes dsts_dev (contents lost)."""
-    handle = stream.cuda_stream if hasattr(stream, "cuda_stream") else stream
-    code = lib().rudra_stream_probe(_ptr_array(srcs_dev) if srcs_dev else None, len(srcs_dev),
-                                    _ptr_array(dsts_dev) if dsts_dev else None, len(dsts_dev), int(nfloats), handle)
-    if code < 0:
-        raise RudraError(code, "rudra_stream_probe refused its arguments or the launch failed")
     return code
 
 

@@ -9,9 +9,18 @@
 
 #include <cuda_runtime.h>
 
-#include "../../include/rudra_ps.h"
-
+// Built into its own shared object (librudra_probe.so) for the benchmark; it is not part of the
+// parameter-server library and not declared in its header.
+//
+//   int rudra_stream_probe(const float* const* srcs_dev, uint32_t nreads, float* const* dsts_dev,
+//                          uint32_t nwrites, uint64_t nfloats, void* cuda_stream);
+//
+// Enqueues one kernel that reads nreads vectors (host array srcs_dev of device pointers) and
+// writes nwrites vectors (dsts_dev; their contents become meaningless), nfloats floats each,
+// 32-byte aligned, at most 64 of each.  Returns 0, -1 for bad arguments, -4 if the launch failed.
 namespace {
+
+constexpr int kBadArgument = -1, kLaunchFailed = -4;
 
 constexpr int kMaxStreams = 64;
 
@@ -62,22 +71,22 @@ __global__ void __launch_bounds__(256) probe_kernel(const __grid_constant__ Prob
 
 extern "C" int rudra_stream_probe(const float* const* srcs_dev, uint32_t nreads, float* const* dsts_dev,
                                   uint32_t nwrites, uint64_t nfloats, void* cuda_stream) {
-  if (nreads > kMaxStreams || nwrites > kMaxStreams || nreads + nwrites == 0 || nfloats < 8) return RUDRA_E_INVAL;
-  if ((nreads && !srcs_dev) || (nwrites && !dsts_dev)) return RUDRA_E_INVAL;
+  if (nreads > kMaxStreams || nwrites > kMaxStreams || nreads + nwrites == 0 || nfloats < 8) return kBadArgument;
+  if ((nreads && !srcs_dev) || (nwrites && !dsts_dev)) return kBadArgument;
   ProbeParams p;
   for (uint32_t i = 0; i < nreads; ++i) {
-    if (!srcs_dev[i] || (reinterpret_cast<uintptr_t>(srcs_dev[i]) & 31)) return RUDRA_E_INVAL;
+    if (!srcs_dev[i] || (reinterpret_cast<uintptr_t>(srcs_dev[i]) & 31)) return kBadArgument;
     p.src[i] = srcs_dev[i];
   }
   for (uint32_t i = 0; i < nwrites; ++i) {
-    if (!dsts_dev[i] || (reinterpret_cast<uintptr_t>(dsts_dev[i]) & 31)) return RUDRA_E_INVAL;
+    if (!dsts_dev[i] || (reinterpret_cast<uintptr_t>(dsts_dev[i]) & 31)) return kBadArgument;
     p.dst[i] = dsts_dev[i];
   }
   p.nunits = nfloats / 8;
   p.nreads = nreads;
   p.nwrites = nwrites;
   const uint64_t blocks = (p.nunits + 255) / 256;
-  if (blocks > 0x7FFFFFFFull) return RUDRA_E_INVAL;
+  if (blocks > 0x7FFFFFFFull) return kBadArgument;
   probe_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
-  return cudaGetLastError() == cudaSuccess ? 0 : RUDRA_E_CUDA;
+  return cudaGetLastError() == cudaSuccess ? 0 : kLaunchFailed;
 }

@@ -33,6 +33,20 @@ int cuda_fail(cudaError_t e, const char* what) {
   return fail(RUDRA_E_CUDA, "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
 }
 
+// Runs the body of an exported function; a C++ exception (in practice std::bad_alloc from a host
+// container) becomes an error code instead of crossing the C boundary.
+template <typename F>
+auto guarded(F&& body) -> decltype(body()) {
+  using R = decltype(body());
+  try {
+    return body();
+  } catch (const std::bad_alloc&) {
+    return (R)fail(RUDRA_E_NOMEM, "out of host memory");
+  } catch (...) {
+    return (R)fail(RUDRA_E_NOMEM, "unexpected C++ exception");
+  }
+}
+
 constexpr uint32_t kMagic = 0x52554452u;   // "RUDR"
 constexpr uintptr_t kAlignMask = 31;       // 256-bit vector accesses
 
@@ -95,6 +109,7 @@ struct rudra_ps {
   // update to keep track of the average staleness): a ring of the last kClockLog updates, c
   // gradient timestamps each, and a histogram of every staleness value seen since create.
   static constexpr uint32_t kClockLog = 4096;
+  static constexpr uint32_t kHistBins = RUDRA_HIST_BINS;
   std::vector<uint64_t> log_pulled;     // kClockLog * c
   std::vector<uint64_t> log_ts;         // timestamp before the update in that ring position, or ~0
   std::vector<uint64_t> sigma_hist;     // count per staleness value, grown on demand
@@ -257,8 +272,11 @@ void append_update(rudra_ps* ps, Window& w) {
     ps->log_ts[pos] = ps->ts;
     for (uint32_t l = 0; l < c; ++l) {
       ps->log_pulled[pos * c + l] = ps->clock[l];
-      if (ps->sigma[l] >= ps->sigma_hist.size()) ps->sigma_hist.resize((size_t)ps->sigma[l] + 1, 0);
-      ps->sigma_hist[ps->sigma[l]] += 1;
+      // the last bin counts every staleness of kHistBins - 1 and more, so one very late gradient
+      // cannot ask for a histogram as long as the timestamp
+      const uint32_t bin = ps->sigma[l] < rudra_ps::kHistBins - 1 ? ps->sigma[l] : rudra_ps::kHistBins - 1;
+      if (bin >= ps->sigma_hist.size()) ps->sigma_hist.resize((size_t)bin + 1, 0);
+      ps->sigma_hist[bin] += 1;
     }
   }
   double sum_scale = 0.0;
@@ -273,8 +291,12 @@ void append_update(rudra_ps* ps, Window& w) {
     sum_scale += (double)ps->scale[l];
   }
   const float abar = (float)sum_scale;
-  for (uint32_t l = 0; l < c; ++l)
-    p.scale[base + l] = ps->optim == RUDRA_OPTIM_ADAGRAD ? (float)((double)ps->scale[l] / (double)abar) : ps->scale[l];
+  for (uint32_t l = 0; l < c; ++l) {
+    // AdaGrad combines the gradients with weights s_l / sum(s); with a zero rate every s_l is 0 and
+    // the weights fall back to Eq. 5's plain 1/c (the weights do not move, the sum of squares does)
+    const float weight = abar > 0.f ? (float)((double)ps->scale[l] / (double)abar) : (float)(1.0 / (double)c);
+    p.scale[base + l] = ps->optim == RUDRA_OPTIM_ADAGRAD ? weight : ps->scale[l];
+  }
   p.awd[w.nupd] = (float)((double)abar * (double)ps->wd);
   p.abar[w.nupd] = abar;
   p.dst_end[w.nupd] = (uint8_t)w.ndst;   // pulls so far belong to the state before this update
@@ -396,7 +418,7 @@ rudra_ps* rudra_ps_create(uint64_t nparams, uint32_t lambda, uint32_t n, float a
     return nullptr;
   }
   rudra_ps* ps = new (std::nothrow) rudra_ps;
-  if (!ps) { fail(RUDRA_E_CUDA, "out of host memory"); return nullptr; }
+  if (!ps) { fail(RUDRA_E_NOMEM, "out of host memory"); return nullptr; }
   ps->N = nparams; ps->lambda = lambda; ps->n = n; ps->c = lambda / n;
   ps->alpha0 = alpha0; ps->momentum = momentum; ps->wd = weight_decay;
   cudaError_t e = cudaGetDevice(&ps->device);
@@ -429,46 +451,52 @@ void rudra_ps_destroy(rudra_ps* ps) {
 }
 
 int rudra_ps_set_stream(rudra_ps* ps, void* cuda_stream) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  ps->stream = static_cast<cudaStream_t>(cuda_stream);
-  return 0;
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    ps->stream = static_cast<cudaStream_t>(cuda_stream);
+    return 0;
+  });
 }
 
 int rudra_ps_set_option(rudra_ps* ps, int key, int64_t value) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (!ps->queue.empty()) return fail(RUDRA_E_STATE, "options can only change while no gradient is queued");
-  DeviceScope dev(ps->device);
-  switch (key) {
-    case RUDRA_OPT_GRAD_DTYPE:
-      if (value != RUDRA_GRAD_F32 && value != RUDRA_GRAD_BF16) return fail(RUDRA_E_INVAL, "unknown gradient type %lld", (long long)value);
-      if ((int)value != ps->gtype) {
-        int r = free_staging(ps);   // staging buffers are sized for the gradient type
-        if (r < 0) return r;
-        ps->gtype = (int)value;
-      }
-      return 0;
-    case RUDRA_OPT_LR_POLICY:
-      if (value < RUDRA_LR_PAPER_N || value > RUDRA_LR_GROUP_MEAN) return fail(RUDRA_E_INVAL, "unknown learning-rate policy %lld", (long long)value);
-      ps->policy = (int)value;
-      return 0;
-    case RUDRA_OPT_OPTIMIZER:
-      if (value != RUDRA_OPTIM_MOMENTUM_SGD && value != RUDRA_OPTIM_ADAGRAD) return fail(RUDRA_E_INVAL, "unknown optimizer %lld", (long long)value);
-      if ((int)value != ps->optim) {
-        cudaError_t e = cudaMemsetAsync(ps->state, 0, ps->N * sizeof(float), ps->stream);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
-        ps->optim = (int)value;
-      }
-      return 0;
-    default:
-      return fail(RUDRA_E_INVAL, "unknown option key %d", key);
-  }
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!ps->queue.empty()) return fail(RUDRA_E_STATE, "options can only change while no gradient is queued");
+    DeviceScope dev(ps->device);
+    switch (key) {
+      case RUDRA_OPT_GRAD_DTYPE:
+        if (value != RUDRA_GRAD_F32 && value != RUDRA_GRAD_BF16) return fail(RUDRA_E_INVAL, "unknown gradient type %lld", (long long)value);
+        if ((int)value != ps->gtype) {
+          int r = free_staging(ps);   // staging buffers are sized for the gradient type
+          if (r < 0) return r;
+          ps->gtype = (int)value;
+        }
+        return 0;
+      case RUDRA_OPT_LR_POLICY:
+        if (value < RUDRA_LR_PAPER_N || value > RUDRA_LR_GROUP_MEAN) return fail(RUDRA_E_INVAL, "unknown learning-rate policy %lld", (long long)value);
+        ps->policy = (int)value;
+        return 0;
+      case RUDRA_OPT_OPTIMIZER:
+        if (value != RUDRA_OPTIM_MOMENTUM_SGD && value != RUDRA_OPTIM_ADAGRAD) return fail(RUDRA_E_INVAL, "unknown optimizer %lld", (long long)value);
+        if ((int)value != ps->optim) {
+          cudaError_t e = cudaMemsetAsync(ps->state, 0, ps->N * sizeof(float), ps->stream);
+          if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+          ps->optim = (int)value;
+        }
+        return 0;
+      default:
+        return fail(RUDRA_E_INVAL, "unknown option key %d", key);
+    }
+  });
 }
 
 int rudra_ps_set_alpha0(rudra_ps* ps, float alpha0) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (!std::isfinite(alpha0) || alpha0 < 0.f) return fail(RUDRA_E_INVAL, "alpha0 must be finite and non-negative");
-  ps->alpha0 = alpha0;
-  return 0;
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!std::isfinite(alpha0) || alpha0 < 0.f) return fail(RUDRA_E_INVAL, "alpha0 must be finite and non-negative");
+    ps->alpha0 = alpha0;
+    return 0;
+  });
 }
 
 static int set_weights_common(rudra_ps* ps, const float* src, cudaMemcpyKind kind) {
@@ -488,382 +516,418 @@ static int set_weights_common(rudra_ps* ps, const float* src, cudaMemcpyKind kin
 }
 
 int rudra_ps_set_weights(rudra_ps* ps, const float* src_dev) {
-  return set_weights_common(ps, src_dev, cudaMemcpyDeviceToDevice);
+  return guarded([&]() -> int { return set_weights_common(ps, src_dev, cudaMemcpyDeviceToDevice); });
 }
 
 int rudra_ps_set_weights_host(rudra_ps* ps, const float* src_host) {
-  return set_weights_common(ps, src_host, cudaMemcpyHostToDevice);
+  return guarded([&]() -> int { return set_weights_common(ps, src_host, cudaMemcpyHostToDevice); });
 }
 
 int64_t rudra_ps_push(rudra_ps* ps, const void* grad_dev, uint64_t pulled_ts) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (!aligned(grad_dev)) return fail(RUDRA_E_INVAL, "gradient pointer is null or not 32-byte aligned");
-  if (int r = check_push(ps, pulled_ts)) return r;
-  return enqueue(ps, grad_dev, pulled_ts, -1);
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!aligned(grad_dev)) return fail(RUDRA_E_INVAL, "gradient pointer is null or not 32-byte aligned");
+    if (int r = check_push(ps, pulled_ts)) return r;
+    return enqueue(ps, grad_dev, pulled_ts, -1);
+  });
 }
 
 int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_ts) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (!grad_host) return fail(RUDRA_E_INVAL, "null gradient pointer");
-  if (int r = check_push(ps, pulled_ts)) return r;
-  DeviceScope dev(ps->device);
-  cudaError_t e = ensure_copy_streams(ps);
-  if (e != cudaSuccess) return cuda_fail(e, "copy stream creation");
-  int slot;
-  if (!ps->free_slots.empty()) {
-    slot = ps->free_slots.back();
-    ps->free_slots.pop_back();
-    e = cudaStreamWaitEvent(ps->up_stream, ps->slot_spent[slot], 0);   // its last reader must be done
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!grad_host) return fail(RUDRA_E_INVAL, "null gradient pointer");
+    if (int r = check_push(ps, pulled_ts)) return r;
+    DeviceScope dev(ps->device);
+    cudaError_t e = ensure_copy_streams(ps);
+    if (e != cudaSuccess) return cuda_fail(e, "copy stream creation");
+    int slot;
+    if (!ps->free_slots.empty()) {
+      slot = ps->free_slots.back();
+      ps->free_slots.pop_back();
+      e = cudaStreamWaitEvent(ps->up_stream, ps->slot_spent[slot], 0);   // its last reader must be done
+      if (e != cudaSuccess) {
+        ps->free_slots.push_back(slot);
+        return cuda_fail(e, "cudaStreamWaitEvent");
+      }
+    } else {
+      void* buf = nullptr;
+      cudaEvent_t ready = nullptr, spent = nullptr;
+      e = cudaMalloc(&buf, ps->grad_bytes());
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ready, cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&spent, cudaEventDisableTiming);
+      if (e != cudaSuccess) {
+        cudaFree(buf);
+        if (ready) cudaEventDestroy(ready);
+        return cuda_fail(e, "staging buffer allocation");
+      }
+      ps->slots.push_back(buf);
+      ps->slot_ready.push_back(ready);
+      ps->slot_spent.push_back(spent);
+      slot = (int)ps->slots.size() - 1;
+    }
+    e = cudaMemcpyAsync(ps->slots[slot], grad_host, ps->grad_bytes(), cudaMemcpyHostToDevice, ps->up_stream);
+    if (e == cudaSuccess) e = cudaEventRecord(ps->slot_ready[slot], ps->up_stream);
     if (e != cudaSuccess) {
       ps->free_slots.push_back(slot);
-      return cuda_fail(e, "cudaStreamWaitEvent");
+      return cuda_fail(e, "gradient host-to-device copy");
     }
-  } else {
-    void* buf = nullptr;
-    cudaEvent_t ready = nullptr, spent = nullptr;
-    e = cudaMalloc(&buf, ps->grad_bytes());
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ready, cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&spent, cudaEventDisableTiming);
-    if (e != cudaSuccess) {
-      cudaFree(buf);
-      if (ready) cudaEventDestroy(ready);
-      return cuda_fail(e, "staging buffer allocation");
-    }
-    ps->slots.push_back(buf);
-    ps->slot_ready.push_back(ready);
-    ps->slot_spent.push_back(spent);
-    slot = (int)ps->slots.size() - 1;
-  }
-  e = cudaMemcpyAsync(ps->slots[slot], grad_host, ps->grad_bytes(), cudaMemcpyHostToDevice, ps->up_stream);
-  if (e == cudaSuccess) e = cudaEventRecord(ps->slot_ready[slot], ps->up_stream);
-  if (e != cudaSuccess) {
-    ps->free_slots.push_back(slot);
-    return cuda_fail(e, "gradient host-to-device copy");
-  }
-  ps->counters[4] += ps->grad_bytes();
-  return enqueue(ps, ps->slots[slot], pulled_ts, slot);
+    ps->counters[4] += ps->grad_bytes();
+    return enqueue(ps, ps->slots[slot], pulled_ts, slot);
+  });
 }
 
-int rudra_ps_step(rudra_ps* ps) { return do_step(ps, nullptr, 0); }
+int rudra_ps_step(rudra_ps* ps) {
+  return guarded([&]() -> int { return do_step(ps, nullptr, 0); });
+}
 
-int rudra_ps_step_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) { return do_step(ps, dsts_dev, k); }
+int rudra_ps_step_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) {
+  return guarded([&]() -> int { return do_step(ps, dsts_dev, k); });
+}
 
 int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t count,
                             const void* const* grads_dev, float* const* slots_dev, uint32_t max_window) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (count && !events) return fail(RUDRA_E_INVAL, "null event list");
-  const uint32_t cap = max_window == 0 || max_window > (uint32_t)rudra::kMaxWindow ? (uint32_t)rudra::kMaxWindow : max_window;
-  // Pass 1: replay the integers only.  Nothing is queued or launched unless the whole batch is legal.
-  const bool views = ps->views_enabled();
-  {
-    uint64_t ts = ps->ts;
-    uint64_t queued = ps->queue.size();
-    ViewBook sim(ps);
-    bool fresh;
-    for (uint64_t i = 0; i < count; ++i) {
-      const rudra_event& ev = events[i];
-      const bool needs_learner = ev.kind == RUDRA_EV_PUSH || ev.kind == RUDRA_EV_PULL;
-      if (needs_learner && ev.learner >= ps->lambda) return fail(RUDRA_E_INVAL, "event %llu: learner %u out of range", (unsigned long long)i, ev.learner);
-      switch (ev.kind) {
-        case RUDRA_EV_PUSH:
-          if (!grads_dev || !aligned(grads_dev[ev.learner])) return fail(RUDRA_E_INVAL, "event %llu: gradient buffer of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
-          if (ev.pulled_ts > ts) return fail(RUDRA_E_BAD_TS, "event %llu: pulled_ts %llu is ahead of the server timestamp %llu", (unsigned long long)i, (unsigned long long)ev.pulled_ts, (unsigned long long)ts);
-          if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: push expects server timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
-          if (++queued > RUDRA_QUEUE_CAP) return fail(RUDRA_E_QUEUE_FULL, "event %llu: queue full", (unsigned long long)i);
-          break;
-        case RUDRA_EV_STEP:
-          if (queued < ps->c) return fail(RUDRA_E_STATE, "event %llu: update with %llu of %u gradients queued", (unsigned long long)i, (unsigned long long)queued, ps->c);
-          queued -= ps->c;
-          ts += 1;
-          if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: update expects new timestamp %llu, server reaches %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
-          break;
-        case RUDRA_EV_PULL:
-          if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: pull expects timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
-          if (views) {
-            if (sim.adopt(ev.learner, ts, &fresh) < 0) return fail(RUDRA_E_STATE, "event %llu: all %zu weight versions are still held by learners", (unsigned long long)i, sim.ts.size());
-          } else if (!slots_dev || !aligned(slots_dev[ev.learner])) {
-            return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
-          }
-          break;
-        case RUDRA_EV_PULL_SKIP:
-          break;
-        case RUDRA_EV_BROADCAST:
-          if (views) {
-            for (uint32_t l = 0; l < ps->lambda; ++l)
-              if (sim.adopt(l, ts, &fresh) < 0) return fail(RUDRA_E_STATE, "event %llu: all %zu weight versions are still held by learners", (unsigned long long)i, sim.ts.size());
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (count && !events) return fail(RUDRA_E_INVAL, "null event list");
+    const uint32_t cap = max_window == 0 || max_window > (uint32_t)rudra::kMaxWindow ? (uint32_t)rudra::kMaxWindow : max_window;
+    // Pass 1: replay the integers only.  Nothing is queued or launched unless the whole batch is legal.
+    const bool views = ps->views_enabled();
+    {
+      uint64_t ts = ps->ts;
+      uint64_t queued = ps->queue.size();
+      ViewBook sim(ps);
+      bool fresh;
+      for (uint64_t i = 0; i < count; ++i) {
+        const rudra_event& ev = events[i];
+        const bool needs_learner = ev.kind == RUDRA_EV_PUSH || ev.kind == RUDRA_EV_PULL;
+        if (needs_learner && ev.learner >= ps->lambda) return fail(RUDRA_E_INVAL, "event %llu: learner %u out of range", (unsigned long long)i, ev.learner);
+        switch (ev.kind) {
+          case RUDRA_EV_PUSH:
+            if (!grads_dev || !aligned(grads_dev[ev.learner])) return fail(RUDRA_E_INVAL, "event %llu: gradient buffer of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
+            if (ev.pulled_ts > ts) return fail(RUDRA_E_BAD_TS, "event %llu: pulled_ts %llu is ahead of the server timestamp %llu", (unsigned long long)i, (unsigned long long)ev.pulled_ts, (unsigned long long)ts);
+            if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: push expects server timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+            if (++queued > RUDRA_QUEUE_CAP) return fail(RUDRA_E_QUEUE_FULL, "event %llu: queue full", (unsigned long long)i);
             break;
-          }
-          if (!slots_dev) return fail(RUDRA_E_INVAL, "event %llu: broadcast without slots", (unsigned long long)i);
-          for (uint32_t l = 0; l < ps->lambda; ++l)
-            if (!aligned(slots_dev[l])) return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, l);
-          break;
-        default:
-          return fail(RUDRA_E_INVAL, "event %llu: unknown kind %d", (unsigned long long)i, ev.kind);
+          case RUDRA_EV_STEP:
+            if (queued < ps->c) return fail(RUDRA_E_STATE, "event %llu: update with %llu of %u gradients queued", (unsigned long long)i, (unsigned long long)queued, ps->c);
+            queued -= ps->c;
+            ts += 1;
+            if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: update expects new timestamp %llu, server reaches %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+            break;
+          case RUDRA_EV_PULL:
+            if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: pull expects timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+            if (views) {
+              if (sim.adopt(ev.learner, ts, &fresh) < 0) return fail(RUDRA_E_STATE, "event %llu: all %zu weight versions are still held by learners", (unsigned long long)i, sim.ts.size());
+            } else if (!slots_dev || !aligned(slots_dev[ev.learner])) {
+              return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
+            }
+            break;
+          case RUDRA_EV_PULL_SKIP:
+            break;
+          case RUDRA_EV_BROADCAST:
+            if (views) {
+              for (uint32_t l = 0; l < ps->lambda; ++l)
+                if (sim.adopt(l, ts, &fresh) < 0) return fail(RUDRA_E_STATE, "event %llu: all %zu weight versions are still held by learners", (unsigned long long)i, sim.ts.size());
+              break;
+            }
+            if (!slots_dev) return fail(RUDRA_E_INVAL, "event %llu: broadcast without slots", (unsigned long long)i);
+            for (uint32_t l = 0; l < ps->lambda; ++l)
+              if (!aligned(slots_dev[l])) return fail(RUDRA_E_INVAL, "event %llu: slot of learner %u is null or not 32-byte aligned", (unsigned long long)i, l);
+            break;
+          default:
+            return fail(RUDRA_E_INVAL, "event %llu: unknown kind %d", (unsigned long long)i, ev.kind);
+        }
       }
     }
-  }
-  // Pass 2: handle the messages in order, packing consecutive updates and the pulls between them
-  // into one launch for as long as the launch tables have room.
-  DeviceScope dev(ps->device);
-  if (!dev.ok()) return fail(RUDRA_E_CUDA, "cannot select device %d", ps->device);
-  Window w;
-  int64_t updates = 0;
-  ViewBook book(ps);
-  auto add_copy = [&](float* dst) -> int {
-    if (w.ndst == (uint32_t)rudra::kMaxDsts)
-      if (int r = flush_window(ps, w)) return r;
-    w.p.dst[w.ndst++] = dst;
-    return 0;
-  };
-  // One learner's pull: a copy into its slot, or (zero-copy mode) a reference to the version with
-  // the current timestamp, which is written at most once however many learners take it.
-  auto add_pull = [&](uint32_t learner) -> int {
-    w.npulls += 1;
-    if (!views) return add_copy(slots_dev[learner]);
-    bool fresh = false;
-    const int idx = book.adopt(learner, ps->ts, &fresh);
-    if (fresh) {
-      if (int r = add_copy(ps->versions[idx].buf)) return r;
-      w.nversions += 1;
+    // Pass 2: handle the messages in order, packing consecutive updates and the pulls between them
+    // into one launch for as long as the launch tables have room.
+    DeviceScope dev(ps->device);
+    if (!dev.ok()) return fail(RUDRA_E_CUDA, "cannot select device %d", ps->device);
+    Window w;
+    int64_t updates = 0;
+    ViewBook book(ps);
+    auto add_copy = [&](float* dst) -> int {
+      if (w.ndst == (uint32_t)rudra::kMaxDsts)
+        if (int r = flush_window(ps, w)) return r;
+      w.p.dst[w.ndst++] = dst;
+      return 0;
+    };
+    // One learner's pull: a copy into its slot, or (zero-copy mode) a reference to the version with
+    // the current timestamp, which is written at most once however many learners take it.
+    auto add_pull = [&](uint32_t learner) -> int {
+      w.npulls += 1;
+      if (!views) return add_copy(slots_dev[learner]);
+      bool fresh = false;
+      const int idx = book.adopt(learner, ps->ts, &fresh);
+      if (fresh) {
+        if (int r = add_copy(ps->versions[idx].buf)) return r;
+        w.nversions += 1;
+      }
+      return 0;
+    };
+    for (uint64_t i = 0; i < count; ++i) {
+      const rudra_event& ev = events[i];
+      switch (ev.kind) {
+        case RUDRA_EV_PUSH:
+          enqueue(ps, grads_dev[ev.learner], ev.pulled_ts, -1);
+          break;
+        case RUDRA_EV_STEP:
+          if (!window_has_room_for_update(ps, w, cap))
+            if (int r = flush_window(ps, w)) return r;
+          append_update(ps, w);
+          updates += 1;
+          break;
+        case RUDRA_EV_PULL:
+          if (int r = add_pull(ev.learner)) return r;
+          break;
+        case RUDRA_EV_BROADCAST:
+          for (uint32_t l = 0; l < ps->lambda; ++l)
+            if (int r = add_pull(l)) return r;
+          break;
+        default:
+          break;
+      }
     }
-    return 0;
-  };
-  for (uint64_t i = 0; i < count; ++i) {
-    const rudra_event& ev = events[i];
-    switch (ev.kind) {
-      case RUDRA_EV_PUSH:
-        enqueue(ps, grads_dev[ev.learner], ev.pulled_ts, -1);
-        break;
-      case RUDRA_EV_STEP:
-        if (!window_has_room_for_update(ps, w, cap))
-          if (int r = flush_window(ps, w)) return r;
-        append_update(ps, w);
-        updates += 1;
-        break;
-      case RUDRA_EV_PULL:
-        if (int r = add_pull(ev.learner)) return r;
-        break;
-      case RUDRA_EV_BROADCAST:
-        for (uint32_t l = 0; l < ps->lambda; ++l)
-          if (int r = add_pull(l)) return r;
-        break;
-      default:
-        break;
-    }
-  }
-  if (views) book.store(ps);
-  if (int r = flush_window(ps, w)) return r;
-  return updates;
+    if (views) book.store(ps);
+    if (int r = flush_window(ps, w)) return r;
+    return updates;
+  });
 }
 
 int rudra_ps_enable_views(rudra_ps* ps, uint32_t nversions) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (nversions < 2 || nversions > 4096) return fail(RUDRA_E_INVAL, "need 2 <= nversions <= 4096");
-  for (int v : ps->view_of)
-    if (v >= 0) return fail(RUDRA_E_STATE, "learners still hold views");
-  DeviceScope dev(ps->device);
-  cudaError_t e = cudaStreamSynchronize(ps->stream);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
-  for (auto& v : ps->versions) cudaFree(v.buf);
-  ps->versions.clear();
-  ps->view_of.assign(ps->lambda, -1);
-  for (uint32_t i = 0; i < nversions; ++i) {
-    rudra_ps::Version v;
-    e = cudaMalloc(reinterpret_cast<void**>(&v.buf), ps->N * sizeof(float));
-    if (e != cudaSuccess) {
-      for (auto& u : ps->versions) cudaFree(u.buf);
-      ps->versions.clear();
-      return cuda_fail(e, "weight version allocation");
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (nversions < 2 || nversions > 4096) return fail(RUDRA_E_INVAL, "need 2 <= nversions <= 4096");
+    for (int v : ps->view_of)
+      if (v >= 0) return fail(RUDRA_E_STATE, "learners still hold views");
+    DeviceScope dev(ps->device);
+    cudaError_t e = cudaStreamSynchronize(ps->stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    for (auto& v : ps->versions) cudaFree(v.buf);
+    ps->versions.clear();
+    ps->view_of.assign(ps->lambda, -1);
+    for (uint32_t i = 0; i < nversions; ++i) {
+      rudra_ps::Version v;
+      e = cudaMalloc(reinterpret_cast<void**>(&v.buf), ps->N * sizeof(float));
+      if (e != cudaSuccess) {
+        for (auto& u : ps->versions) cudaFree(u.buf);
+        ps->versions.clear();
+        return cuda_fail(e, "weight version allocation");
+      }
+      ps->versions.push_back(v);
     }
-    ps->versions.push_back(v);
-  }
-  return 0;
+    return 0;
+  });
 }
 
 int64_t rudra_ps_pull_view(rudra_ps* ps, uint32_t learner, const float** view_out) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (!ps->views_enabled()) return fail(RUDRA_E_STATE, "call rudra_ps_enable_views first");
-  if (learner >= ps->lambda || !view_out) return fail(RUDRA_E_INVAL, "learner out of range or null output");
-  ViewBook book(ps);
-  bool fresh = false;
-  const int idx = book.adopt(learner, ps->ts, &fresh);
-  if (idx < 0) return fail(RUDRA_E_STATE, "all %zu weight versions are still held by learners", ps->versions.size());
-  DeviceScope dev(ps->device);
-  Window w;
-  w.npulls = 1;
-  if (fresh) {
-    w.p.dst[w.ndst++] = ps->versions[idx].buf;
-    w.nversions = 1;
-  }
-  book.store(ps);
-  if (int r = flush_window(ps, w)) return r;   // a snapshot launch if the version is new
-  *view_out = ps->versions[idx].buf;
-  return (int64_t)ps->ts;
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!ps->views_enabled()) return fail(RUDRA_E_STATE, "call rudra_ps_enable_views first");
+    if (learner >= ps->lambda || !view_out) return fail(RUDRA_E_INVAL, "learner out of range or null output");
+    ViewBook book(ps);
+    bool fresh = false;
+    const int idx = book.adopt(learner, ps->ts, &fresh);
+    if (idx < 0) return fail(RUDRA_E_STATE, "all %zu weight versions are still held by learners", ps->versions.size());
+    DeviceScope dev(ps->device);
+    Window w;
+    w.npulls = 1;
+    if (fresh) {
+      w.p.dst[w.ndst++] = ps->versions[idx].buf;
+      w.nversions = 1;
+    }
+    book.store(ps);
+    if (int r = flush_window(ps, w)) return r;   // a snapshot launch if the version is new
+    *view_out = ps->versions[idx].buf;
+    return (int64_t)ps->ts;
+  });
 }
 
 int64_t rudra_ps_view_of(const rudra_ps* ps, uint32_t learner, const float** view_out) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (!ps->views_enabled() || learner >= ps->lambda || !view_out) return fail(RUDRA_E_INVAL, "views not enabled, learner out of range or null output");
-  const int idx = ps->view_of[learner];
-  if (idx < 0) return fail(RUDRA_E_STATE, "learner %u holds no view", learner);
-  *view_out = ps->versions[idx].buf;
-  return (int64_t)ps->versions[idx].ts;
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!ps->views_enabled() || learner >= ps->lambda || !view_out) return fail(RUDRA_E_INVAL, "views not enabled, learner out of range or null output");
+    const int idx = ps->view_of[learner];
+    if (idx < 0) return fail(RUDRA_E_STATE, "learner %u holds no view", learner);
+    *view_out = ps->versions[idx].buf;
+    return (int64_t)ps->versions[idx].ts;
+  });
 }
 
 int64_t rudra_ps_pull_many(rudra_ps* ps, float* const* dsts_dev, uint32_t k) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (k == 0) return (int64_t)ps->ts;
-  if (k > RUDRA_MAX_DSTS) return fail(RUDRA_E_INVAL, "k = %u exceeds RUDRA_MAX_DSTS", k);
-  if (!dsts_dev) return fail(RUDRA_E_INVAL, "null destination list");
-  rudra::SnapshotParams p;
-  for (uint32_t d = 0; d < k; ++d) {
-    if (!aligned(dsts_dev[d])) return fail(RUDRA_E_INVAL, "destination %u is null or not 32-byte aligned", d);
-    p.dst[d] = dsts_dev[d];
-  }
-  p.src = ps->theta;
-  p.n = ps->N;
-  p.ndst = k;
-  p.reverse = ps->sweep++ & 1u;
-  DeviceScope dev(ps->device);
-  cudaError_t e = rudra::launch_snapshot(p, ps->stream);
-  if (e != cudaSuccess) return cuda_fail(e, "snapshot kernel launch");
-  ps->counters[2] += k;
-  ps->counters[3] += 1;
-  ps->counters[6] += k;
-  return (int64_t)ps->ts;
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (k == 0) return (int64_t)ps->ts;
+    if (k > RUDRA_MAX_DSTS) return fail(RUDRA_E_INVAL, "k = %u exceeds RUDRA_MAX_DSTS", k);
+    if (!dsts_dev) return fail(RUDRA_E_INVAL, "null destination list");
+    rudra::SnapshotParams p;
+    for (uint32_t d = 0; d < k; ++d) {
+      if (!aligned(dsts_dev[d])) return fail(RUDRA_E_INVAL, "destination %u is null or not 32-byte aligned", d);
+      p.dst[d] = dsts_dev[d];
+    }
+    p.src = ps->theta;
+    p.n = ps->N;
+    p.ndst = k;
+    p.reverse = ps->sweep++ & 1u;
+    DeviceScope dev(ps->device);
+    cudaError_t e = rudra::launch_snapshot(p, ps->stream);
+    if (e != cudaSuccess) return cuda_fail(e, "snapshot kernel launch");
+    ps->counters[2] += k;
+    ps->counters[3] += 1;
+    ps->counters[6] += k;
+    return (int64_t)ps->ts;
+  });
 }
 
 int64_t rudra_ps_pull(rudra_ps* ps, float* dst_dev) { return rudra_ps_pull_many(ps, &dst_dev, 1); }
 
 int64_t rudra_ps_pull_host(rudra_ps* ps, float* dst_host) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (!dst_host) return fail(RUDRA_E_INVAL, "null destination");
-  DeviceScope dev(ps->device);
-  cudaError_t e = ensure_copy_streams(ps);
-  if (e != cudaSuccess) return cuda_fail(e, "copy stream creation");
-  constexpr uint32_t kDownBufs = 4;   // snapshots that may be on their way to the host at once
-  if (ps->down.size() < kDownBufs) {
-    rudra_ps::DownBuf d;
-    e = cudaMalloc(reinterpret_cast<void**>(&d.buf), ps->N * sizeof(float));
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&d.filled, cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&d.drained, cudaEventDisableTiming);
-    if (e != cudaSuccess) {
-      cudaFree(d.buf);
-      if (d.filled) cudaEventDestroy(d.filled);
-      return cuda_fail(e, "snapshot buffer allocation");
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!dst_host) return fail(RUDRA_E_INVAL, "null destination");
+    DeviceScope dev(ps->device);
+    cudaError_t e = ensure_copy_streams(ps);
+    if (e != cudaSuccess) return cuda_fail(e, "copy stream creation");
+    constexpr uint32_t kDownBufs = 4;   // snapshots that may be on their way to the host at once
+    if (ps->down.size() < kDownBufs) {
+      rudra_ps::DownBuf d;
+      e = cudaMalloc(reinterpret_cast<void**>(&d.buf), ps->N * sizeof(float));
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&d.filled, cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&d.drained, cudaEventDisableTiming);
+      if (e != cudaSuccess) {
+        cudaFree(d.buf);
+        if (d.filled) cudaEventDestroy(d.filled);
+        return cuda_fail(e, "snapshot buffer allocation");
+      }
+      ps->down.push_back(d);
     }
-    ps->down.push_back(d);
-  }
-  rudra_ps::DownBuf& d = ps->down[ps->down_next++ % ps->down.size()];
-  // snapshot on the main stream (after every update issued so far), then the copy to the host
-  // on the download stream, so later updates need not wait for PCIe
-  e = cudaStreamWaitEvent(ps->stream, d.drained, 0);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent");
-  rudra::SnapshotParams sp;
-  sp.dst[0] = d.buf;
-  sp.src = ps->theta;
-  sp.n = ps->N;
-  sp.ndst = 1;
-  sp.reverse = ps->sweep++ & 1u;
-  e = rudra::launch_snapshot(sp, ps->stream);
-  if (e == cudaSuccess) e = cudaEventRecord(d.filled, ps->stream);
-  if (e == cudaSuccess) e = cudaStreamWaitEvent(ps->down_stream, d.filled, 0);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dst_host, d.buf, ps->N * sizeof(float), cudaMemcpyDeviceToHost, ps->down_stream);
-  if (e == cudaSuccess) e = cudaEventRecord(d.drained, ps->down_stream);
-  if (e != cudaSuccess) return cuda_fail(e, "weights device-to-host copy");
-  ps->counters[2] += 1;
-  ps->counters[3] += 1;
-  ps->counters[5] += ps->N * sizeof(float);
-  ps->counters[6] += 1;
-  return (int64_t)ps->ts;
+    rudra_ps::DownBuf& d = ps->down[ps->down_next++ % ps->down.size()];
+    // snapshot on the main stream (after every update issued so far), then the copy to the host
+    // on the download stream, so later updates need not wait for PCIe
+    e = cudaStreamWaitEvent(ps->stream, d.drained, 0);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent");
+    rudra::SnapshotParams sp;
+    sp.dst[0] = d.buf;
+    sp.src = ps->theta;
+    sp.n = ps->N;
+    sp.ndst = 1;
+    sp.reverse = ps->sweep++ & 1u;
+    e = rudra::launch_snapshot(sp, ps->stream);
+    if (e == cudaSuccess) e = cudaEventRecord(d.filled, ps->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ps->down_stream, d.filled, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dst_host, d.buf, ps->N * sizeof(float), cudaMemcpyDeviceToHost, ps->down_stream);
+    if (e == cudaSuccess) e = cudaEventRecord(d.drained, ps->down_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "weights device-to-host copy");
+    ps->counters[2] += 1;
+    ps->counters[3] += 1;
+    ps->counters[5] += ps->N * sizeof(float);
+    ps->counters[6] += 1;
+    return (int64_t)ps->ts;
+  });
 }
 
 int64_t rudra_ps_timestamp(const rudra_ps* ps) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  return (int64_t)ps->ts;
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    return (int64_t)ps->ts;
+  });
 }
 
 int rudra_ps_last_clock(const rudra_ps* ps, uint64_t* pulled_ts_out, uint32_t* sigma_out, float* scale_out,
                         double* avg_sigma_out) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  if (!ps->has_clock) return 0;
-  for (uint32_t l = 0; l < ps->c; ++l) {
-    if (pulled_ts_out) pulled_ts_out[l] = ps->clock[l];
-    if (sigma_out) sigma_out[l] = ps->sigma[l];
-    if (scale_out) scale_out[l] = ps->scale[l];
-  }
-  if (avg_sigma_out) *avg_sigma_out = ps->avg_sigma;
-  return (int)ps->c;
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!ps->has_clock) return 0;
+    for (uint32_t l = 0; l < ps->c; ++l) {
+      if (pulled_ts_out) pulled_ts_out[l] = ps->clock[l];
+      if (sigma_out) sigma_out[l] = ps->sigma[l];
+      if (scale_out) scale_out[l] = ps->scale[l];
+    }
+    if (avg_sigma_out) *avg_sigma_out = ps->avg_sigma;
+    return (int)ps->c;
+  });
 }
 
 int64_t rudra_ps_clock_log(const rudra_ps* ps, uint64_t first_ts, uint64_t count, uint64_t* pulled_ts_out,
                            double* avg_sigma_out) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  uint64_t got = 0;
-  for (; got < count; ++got) {
-    const uint64_t t = first_ts + got;
-    if (t >= ps->ts || ps->log_ts.empty()) break;
-    const size_t pos = (size_t)(t % rudra_ps::kClockLog);
-    if (ps->log_ts[pos] != t) {
-      if (got == 0) return fail(RUDRA_E_STATE, "update %llu is no longer in the log (the last %u are kept)", (unsigned long long)t, rudra_ps::kClockLog);
-      break;
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    uint64_t got = 0;
+    for (; got < count; ++got) {
+      const uint64_t t = first_ts + got;
+      if (t >= ps->ts || ps->log_ts.empty()) break;
+      const size_t pos = (size_t)(t % rudra_ps::kClockLog);
+      if (ps->log_ts[pos] != t) {
+        if (got == 0) return fail(RUDRA_E_STATE, "update %llu is no longer in the log (the last %u are kept)", (unsigned long long)t, rudra_ps::kClockLog);
+        break;
+      }
+      uint64_t sum = 0;
+      for (uint32_t l = 0; l < ps->c; ++l) {
+        const uint64_t p = ps->log_pulled[pos * ps->c + l];
+        if (pulled_ts_out) pulled_ts_out[got * ps->c + l] = p;
+        sum += p;
+      }
+      if (avg_sigma_out) avg_sigma_out[got] = (double)t - (double)sum / (double)ps->c;
     }
-    uint64_t sum = 0;
-    for (uint32_t l = 0; l < ps->c; ++l) {
-      const uint64_t p = ps->log_pulled[pos * ps->c + l];
-      if (pulled_ts_out) pulled_ts_out[got * ps->c + l] = p;
-      sum += p;
-    }
-    if (avg_sigma_out) avg_sigma_out[got] = (double)t - (double)sum / (double)ps->c;
-  }
-  return (int64_t)got;
+    return (int64_t)got;
+  });
 }
 
 int64_t rudra_ps_staleness_histogram(const rudra_ps* ps, uint64_t* counts_out, uint32_t nbins) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  for (uint32_t b = 0; b < nbins && counts_out; ++b) counts_out[b] = b < ps->sigma_hist.size() ? ps->sigma_hist[b] : 0;
-  return (int64_t)ps->sigma_hist.size();
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    for (uint32_t b = 0; b < nbins && counts_out; ++b) counts_out[b] = b < ps->sigma_hist.size() ? ps->sigma_hist[b] : 0;
+    return (int64_t)ps->sigma_hist.size();
+  });
 }
 
 int rudra_ps_export_state(rudra_ps* ps, float* theta_dst_dev, float* state_dst_dev) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  DeviceScope dev(ps->device);
-  cudaError_t e = cudaSuccess;
-  if (theta_dst_dev) e = cudaMemcpyAsync(theta_dst_dev, ps->theta, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
-  if (e == cudaSuccess && state_dst_dev)
-    e = cudaMemcpyAsync(state_dst_dev, ps->state, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
-  if (e != cudaSuccess) return cuda_fail(e, "rudra_ps_export_state");
-  return 0;
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    DeviceScope dev(ps->device);
+    cudaError_t e = cudaSuccess;
+    if (theta_dst_dev) e = cudaMemcpyAsync(theta_dst_dev, ps->theta, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
+    if (e == cudaSuccess && state_dst_dev)
+      e = cudaMemcpyAsync(state_dst_dev, ps->state, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
+    if (e != cudaSuccess) return cuda_fail(e, "rudra_ps_export_state");
+    return 0;
+  });
 }
 
 int rudra_ps_import_state(rudra_ps* ps, const float* theta_src_dev, const float* state_src_dev, uint64_t ts) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  DeviceScope dev(ps->device);
-  cudaError_t e = cudaSuccess;
-  if (theta_src_dev) e = cudaMemcpyAsync(ps->theta, theta_src_dev, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
-  if (e == cudaSuccess && state_src_dev)
-    e = cudaMemcpyAsync(ps->state, state_src_dev, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
-  if (e != cudaSuccess) return cuda_fail(e, "rudra_ps_import_state");
-  release_queue(ps);
-  ps->ts = ts;
-  ps->has_clock = false;
-  for (auto& v : ps->versions) v.valid = false;
-  std::fill(ps->log_ts.begin(), ps->log_ts.end(), ~0ull);
-  return 0;
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    DeviceScope dev(ps->device);
+    cudaError_t e = cudaSuccess;
+    if (theta_src_dev) e = cudaMemcpyAsync(ps->theta, theta_src_dev, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
+    if (e == cudaSuccess && state_src_dev)
+      e = cudaMemcpyAsync(ps->state, state_src_dev, ps->N * sizeof(float), cudaMemcpyDeviceToDevice, ps->stream);
+    if (e != cudaSuccess) return cuda_fail(e, "rudra_ps_import_state");
+    release_queue(ps);
+    ps->ts = ts;
+    ps->has_clock = false;
+    for (auto& v : ps->versions) v.valid = false;
+    std::fill(ps->log_ts.begin(), ps->log_ts.end(), ~0ull);
+    return 0;
+  });
 }
 
 int rudra_ps_sync(rudra_ps* ps) {
-  if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
-  DeviceScope dev(ps->device);
-  cudaError_t e = sync_all(ps);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
-  return 0;
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    DeviceScope dev(ps->device);
+    cudaError_t e = sync_all(ps);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    return 0;
+  });
 }
 
 int rudra_ps_counters(const rudra_ps* ps, uint64_t out[8]) {
-  if (!valid(ps) || !out) return fail(RUDRA_E_INVAL, "bad handle or null output");
-  std::memcpy(out, ps->counters, sizeof(ps->counters));
-  return 0;
+  return guarded([&]() -> int {
+    if (!valid(ps) || !out) return fail(RUDRA_E_INVAL, "bad handle or null output");
+    std::memcpy(out, ps->counters, sizeof(ps->counters));
+    return 0;
+  });
 }
 
 }  // extern "C"

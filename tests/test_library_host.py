@@ -33,13 +33,25 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(L, name), name
 
 
+def test_library_exports_nothing_but_its_interface():
+    import subprocess
+
+    out = subprocess.check_output(["nm", "-D", "--defined-only", rb.library_path()], text=True)
+    exported = {line.split()[-1] for line in out.splitlines() if " T " in line}
+    declared = set(_declared_symbols())
+    extra = sorted(n for n in exported if n.startswith("rudra") and n not in declared)
+    assert not extra, extra                       # e.g. the benchmark's probe lives in a library of its own
+
+
 def test_header_constants_match_binding():
     text = open(os.path.join(ROOT, "include", "rudra_ps.h")).read()
     defs = {k: int(v.strip("()")) for k, v in re.findall(r"#define\s+(RUDRA_[A-Z0-9_]+)\s+(\(?-?\d+\)?)", text)}
     assert defs["RUDRA_MAX_GROUP"] == rb.MAX_GROUP and defs["RUDRA_MAX_DSTS"] == rb.MAX_DSTS
     assert defs["RUDRA_QUEUE_CAP"] == rb.QUEUE_CAP
     assert (defs["RUDRA_E_INVAL"], defs["RUDRA_E_BAD_TS"], defs["RUDRA_E_QUEUE_FULL"], defs["RUDRA_E_CUDA"],
-            defs["RUDRA_E_STATE"]) == (rb.E_INVAL, rb.E_BAD_TS, rb.E_QUEUE_FULL, rb.E_CUDA, rb.E_STATE)
+            defs["RUDRA_E_STATE"], defs["RUDRA_E_NOMEM"]) == (rb.E_INVAL, rb.E_BAD_TS, rb.E_QUEUE_FULL, rb.E_CUDA, rb.E_STATE,
+                                                             rb.E_NOMEM)
+    assert defs["RUDRA_HIST_BINS"] == rb.HIST_BINS
     assert (defs["RUDRA_EV_PUSH"], defs["RUDRA_EV_STEP"], defs["RUDRA_EV_PULL"], defs["RUDRA_EV_PULL_SKIP"],
             defs["RUDRA_EV_BROADCAST"]) == (1, 2, 3, 4, 5)
     assert defs["RUDRA_GRAD_BF16"] == rb.GRAD_BF16 == synth.GRAD_BF16

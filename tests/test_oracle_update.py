@@ -432,6 +432,25 @@ def test_adagrad_brute_force_on_a_tiny_vector():
     assert np.abs(no_wd - want_th).max() > 50 * F32_EPS * np.abs(want_th).max()
 
 
+def test_zero_rate_leaves_the_weights_where_they_are():
+    # alpha0 = 0 makes every step size 0 (Eq. 6): neither optimizer may move a weight, and nothing
+    # may turn into NaN.  AdaGrad's sum of squares still grows, by the square of Eq. 5's plain mean.
+    N = 9
+    gs = [synth.gradient(N, l, 0, 1e-2) for l in range(3)]
+    for opt in (ora.OPT_MOMENTUM_SGD, ora.OPT_ADAGRAD):
+        ps, th0 = _mk(N, 3, 1, 0.0, m=0.9 if opt == ora.OPT_MOMENTUM_SGD else 0.0)
+        ps.set_optimizer(opt, 1e-8)
+        for g in gs:
+            ps.push(g, 0)
+        assert ps.step() == 1
+        np.testing.assert_array_equal(ps.pull()[0], th0.astype(np.float32))
+        if opt == ora.OPT_ADAGRAD:
+            mean = np.mean(np.stack(gs).astype(np.float64), axis=0)
+            _close(ps.state(), mean * mean, 0.0, ulps=4)
+        else:
+            np.testing.assert_array_equal(ps.state(), np.zeros(N, dtype=np.float32))
+
+
 def test_strict_fp32_mode_tracks_the_double_mode():
     # the fp32 evaluation is the same rule: after a few updates it differs only by fp32 rounding
     N, lam, n = 500, 6, 2
