@@ -403,3 +403,37 @@ def test_a_learner_that_never_pushes():
     hard.push(g[3], 0)
     assert hard.step() == 1
     soft.close(), hard.close()
+
+
+@pytest.mark.parametrize("optimizer", [ora.OPT_MOMENTUM_SGD, ora.OPT_ADAGRAD])
+def test_zero_rate_moves_no_weight(optimizer):
+    # alpha0 = 0: every step size is 0 (Eq. 6); the weights stay bit for bit, nothing becomes NaN
+    N = 300011
+    pair = Pair(N, 3, 1, 0.0, 0.9 if optimizer == ora.OPT_MOMENTUM_SGD else 0.0, 5e-4, optimizer=optimizer)
+    for k in range(2):
+        for l in range(3):
+            pair.push(synth.gradient(N, l, k, 1e-2), pair.gpu.timestamp())
+        assert pair.step() == 1
+    th, st = pair.weights()
+    np.testing.assert_array_equal(th, pair.theta0)
+    assert np.isfinite(st).all()
+    pair.compare(REL_ONE_STEP)
+    pair.close()
+
+
+def test_one_very_late_gradient_does_not_grow_the_histogram():
+    from paper_1509_04210_b200 import binding as rb
+
+    N = 64
+    ps = rb.ParameterServer(N, 1, 1, 0.01)
+    g = to_device(synth.gradient(N, 0, 0))
+    th = to_device(synth.initial_weights(N))
+    ps.import_state(th, None, 10**9)               # a server that has been running for a long time
+    ps.push(g, 0)                                   # a gradient from the very first weights
+    assert ps.step() == 1
+    ps.push(g, 10**9 + 1)
+    assert ps.step() == 1
+    hist = ps.staleness_histogram()
+    assert len(hist) == rb.HIST_BINS and hist[-1] == 1 and hist[0] == 1 and hist.sum() == 2
+    assert ps.last_clock()["sigma"][0] == 0
+    ps.close()

@@ -1,15 +1,18 @@
-"""The no-allocation entry point against the regular host-buffer path, through the C interface.
+"""The no-allocation entry point, through the C interface, against the CPU oracle and against the
+regular host-buffer path.
 
 rudra_ps_update_host_noalloc serves callers that cannot allocate device memory while running
 (their own pool owns the GPU, or an allocation's device-wide synchronisation is not acceptable):
 it stages gradients in a fixed array inside the library instead of buffers allocated on demand.
-The update it performs must equal what rudra_ps_push_host + rudra_ps_step produce from the same
-host gradients and step sizes, on two calls in a row (the second re-uses the shared array).
+The update it performs must be the oracle's update within the one-step tolerance, bit for bit the
+oracle's fp32 evaluation, and bit for bit what rudra_ps_push_host + rudra_ps_step produce from the
+same host gradients and step sizes -- on two calls in a row (the second re-uses the shared array).
 This file sorts last so that a run stopping at the first failure has already run every other test.
 """
 import numpy as np
 import pytest
 
+from oracle import rudra_oracle as ora
 from paper_1509_04210_b200 import synth
 
 from helpers import REL_ONE_STEP, rel_err
@@ -17,40 +20,62 @@ from helpers import REL_ONE_STEP, rel_err
 pytestmark = pytest.mark.gpu
 
 
-def test_no_alloc_update_matches_push_host_and_step_twice():
+# N = 100 003 runs the one-weight-per-thread kernel; 300 011 and 1 000 003 run the 256-bit kernel on
+# slots carved from the fixed array (ragged last tile, N % 8 scalar tail, slot stride rounded up
+# to 64 floats); the last case has no momentum and passes no state vector.
+@pytest.mark.parametrize("N,c,m", [(100003, 3, 0.9), (300011, 3, 0.9), (1000003, 3, 0.9), (300011, 2, 0.0)])
+def test_no_alloc_update_matches_oracle_and_host_path_twice(N, c, m):
     import torch
     from paper_1509_04210_b200 import binding as rb
 
-    N, c, m, wd = 100003, 3, 0.9, 5e-4
+    wd, a0 = 5e-4, 0.05
     th0 = synth.initial_weights(N, 0.01, 77)
-    ps = rb.ParameterServer(N, c, 1, 0.05, m, wd)
+    ps = rb.ParameterServer(N, c, 1, a0, m, wd)
     ps.set_option(rb.OPT_LR_POLICY, rb.LR_PER_GRADIENT)
     ps.set_weights_host(np.ascontiguousarray(th0))
+    cpu, strict = ora.OraclePS(N, c, 1, a0, m, wd), ora.OraclePS(N, c, 1, a0, m, wd)
+    for o in (cpu, strict):
+        o.set_policy(ora.LR_PER_GRADIENT)
+        o.set_weights(th0)
+    strict.set_strict(True)
     for warm in range(2):                                    # raise the timestamp so staleness can vary
         for l in range(c):
-            ps.push_host(synth.gradient(N, l, 10 + warm, 1e-2, seed=5), ps.timestamp())
-        assert ps.step() == 1
+            g = synth.gradient(N, l, 10 + warm, 1e-2, seed=5)
+            ps.push_host(g, ps.timestamp())
+            cpu.push(g, cpu.timestamp()), strict.push(g, strict.timestamp())
+        assert ps.step() == 1 and cpu.step() == 1 and strict.step() == 1
     theta = torch.empty(N, device="cuda")
     state = torch.empty(N, device="cuda")
     ps.export_state(theta, state)
     ps.sync()
     want_th = torch.empty(N, device="cuda")
     want_st = torch.empty(N, device="cuda")
+    backs = (0, 2, 1)[:c]                                    # staleness 0, 2, 1: different step sizes
     for call in range(2):
         grads = [synth.gradient(N, l, call, 1e-2, seed=5) for l in range(c)]
         ts = ps.timestamp()
-        for g, back in zip(grads, (0, 2, 1)):                # staleness 0, 2, 1: three different step sizes
+        for g, back in zip(grads, backs):
             ps.push_host(g, ts - back)
-        assert ps.step() == 1
-        assert list(ps.last_clock()["sigma"]) == [0, 2, 1]
+            cpu.push(g, ts - back), strict.push(g, ts - back)
+        assert ps.step() == 1 and cpu.step() == 1 and strict.step() == 1
+        assert list(ps.last_clock()["sigma"]) == list(backs) == list(cpu.last_clock()["sigma"])
         scales = ps.last_clock()["scale"]
+        np.testing.assert_array_equal(scales.view(np.uint32), cpu.last_clock()["scale"].view(np.uint32))
         ps.export_state(want_th, want_st)
         ps.sync()
-        assert rb.update_host_noalloc(theta, state, N, grads, scales, m, wd) == 0
+        assert rb.update_host_noalloc(theta, state if m else None, N, grads, scales, m, wd) == 0
         torch.cuda.synchronize()
-        e_th = rel_err(theta.cpu().numpy(), want_th.cpu().numpy())
-        e_st = rel_err(state.cpu().numpy(), want_st.cpu().numpy())
-        assert e_th <= REL_ONE_STEP and e_st <= REL_ONE_STEP, (call, e_th, e_st)
+        got_th, got_st = theta.cpu().numpy(), state.cpu().numpy()
+        # the oracle: double arithmetic within the tolerance, fp32 evaluation bit for bit
+        assert rel_err(got_th, cpu.pull()[0]) <= REL_ONE_STEP
+        np.testing.assert_array_equal(got_th, strict.pull()[0])
+        if m:
+            assert rel_err(got_st, cpu.state()) <= REL_ONE_STEP
+            np.testing.assert_array_equal(got_st, strict.state())
+        # the same kernel on allocated staging buffers: identical bits
+        assert torch.equal(theta, want_th)
+        if m:
+            assert torch.equal(state, want_st)
     ps.close()
 
 
