@@ -23,6 +23,14 @@
 //     reading at OraclePS::step is pinned by the direction of the first step
 //     (the sign of gradient plus penalty), by a decay-only scalar recurrence
 //     and by brute force in decimal arithmetic with unequal per-gradient rates.
+//   * Rudra-adv's server tree (Section 3.3 says that a leaf averages its
+//     learners' gradients and relays the average to its parent, and that the
+//     root applies the update; it does not say when a leaf relays, which
+//     timestamp a relayed average carries or which rate it gets)
+//                                           : parity unpinned by the paper; the
+//     reading at OraclePS::push_relay is pinned by its reduction to the flat
+//     server (fan-in 1 bit for bit; equal rates to rounding, Eq. 7's argument)
+//     and by hand-computed step sizes.
 // Everything else is pinned by Eq. 2-6 and the staleness sets printed in
 // Section 5.1 (see tests/).
 //
@@ -67,6 +75,7 @@ enum EventKind : int32_t {
   EV_PULL = 3,       // learner receives the weights; ts = their timestamp
   EV_PULL_SKIP = 4,  // timestamp inquiry found the learner's copy current (Section 3.2)
   EV_BROADCAST = 5,  // every learner receives the weights with timestamp ts
+  EV_RELAY = 6,      // tree (Section 3.3): leaf `learner` sends the average of its last k gradients to the root
 };
 
 enum SchedMode : int32_t {
@@ -95,10 +104,17 @@ struct OracleSched {
   bool downcast;          // weights broadcast to every learner after each update (Section 3.3)
   double ln_sigma;
   uint64_t ts = 0;        // server timestamp, starts at 0 (Section 3.1)
-  uint64_t pushes = 0;    // gradients handled so far
+  uint64_t pushes = 0;    // gradients that have reached the (root) server so far
+  // Server tree of Section 3.3, two levels: learner l sends to leaf l / fanin; a leaf that holds
+  // fanin gradients relays their average to the root at once.  fanin = 0: no tree, learners
+  // send to the server directly.
+  uint32_t fanin = 0;
+  std::vector<uint32_t> leaf_fill;   // gradients waiting at each leaf
+  std::vector<uint64_t> leaf_relays; // averages each leaf has relayed
   std::vector<uint64_t> local_ts;   // timestamp of the weights last delivered to each learner
   std::vector<uint64_t> grad_ts;    // timestamp of the weights its current mini-batch started from
   std::vector<uint64_t> nbatch;     // mini-batches each learner has pushed
+  uint64_t handled = 0;             // push messages handled so far (rounds mode: the event tick)
   std::deque<Event> out;
   // rounds
   SplitMix64 perm_rng;
@@ -106,8 +122,10 @@ struct OracleSched {
   std::vector<SplitMix64> time_rng;
   std::vector<uint64_t> next_push;
 
-  OracleSched(uint32_t lambda_, uint32_t n_, int32_t mode_, uint64_t seed, double ln_sigma_, bool downcast_)
+  OracleSched(uint32_t lambda_, uint32_t n_, int32_t mode_, uint64_t seed, double ln_sigma_, bool downcast_,
+              uint32_t fanin_ = 0)
       : lambda(lambda_), n(n_), c(lambda_ / n_), mode(mode_), downcast(downcast_), ln_sigma(ln_sigma_),
+        fanin(fanin_), leaf_fill(fanin_ ? lambda_ / fanin_ : 0, 0), leaf_relays(fanin_ ? lambda_ / fanin_ : 0, 0),
         local_ts(lambda_, 0), grad_ts(lambda_, 0), nbatch(lambda_, 0), perm_rng(stream_state(seed, 1, 0)) {
     if (mode == MODE_SOFTSYNC_TIMED) {
       for (uint32_t l = 0; l < lambda; ++l) time_rng.emplace_back(stream_state(seed, 2, l));
@@ -136,9 +154,21 @@ struct OracleSched {
   void handle_push(uint32_t l, uint64_t tick) {
     emit(EV_PUSH, l, grad_ts[l], ts, nbatch[l], tick);
     nbatch[l] += 1;
-    pushes += 1;
+    bool arrived = true;            // did gradients reach the root with this message?
+    if (fanin == 0) {
+      pushes += 1;
+    } else {
+      const uint32_t leaf = l / fanin;
+      if (++leaf_fill[leaf] == fanin) {   // the leaf averages what it holds and relays it (Section 3.3)
+        leaf_fill[leaf] = 0;
+        emit(EV_RELAY, leaf, 0, ts, leaf_relays[leaf]++, tick);
+        pushes += fanin;            // the average stands for fanin gradients
+      } else {
+        arrived = false;
+      }
+    }
     bool stepped = false;
-    if (pushes % c == 0) {          // exactly c gradients per update (Eq. 5)
+    if (arrived && pushes % c == 0) {   // exactly c gradients per update (Eq. 5)
       ts += 1;                      // one increment per weight update (Section 3.1)
       stepped = true;
       emit(EV_STEP, l, 0, ts, 0, tick);
@@ -182,7 +212,7 @@ struct OracleSched {
       uint32_t j = (uint32_t)(perm_rng.next() % (uint64_t)(i + 1));
       std::swap(perm[i], perm[j]);
     }
-    for (uint32_t i = 0; i < lambda; ++i) handle_push(perm[i], pushes + 1);
+    for (uint32_t i = 0; i < lambda; ++i) handle_push(perm[i], ++handled);
   }
 
   Event next() {
@@ -200,9 +230,14 @@ enum LrPolicy : int32_t { LR_PAPER_N = 0, LR_PER_GRADIENT = 1, LR_GROUP_MEAN = 2
 enum GradDtype : int32_t { GRAD_F32 = 0, GRAD_BF16 = 1 };
 enum Optimizer : int32_t { OPT_MOMENTUM_SGD = 0, OPT_ADAGRAD = 1 };
 
-struct Pending {
-  const void* grad;
-  uint64_t pulled_ts;
+// One message in the server's queue: a learner's gradient (fan-in 1), or the average that a
+// leaf of the server tree relays for `fanin` of its learners' gradients (Section 3.3).  Either
+// way it carries the timestamp of every gradient it stands for.
+struct Message {
+  const void* grad = nullptr;        // fan-in 1: the learner's buffer (borrowed)
+  std::vector<float> avg;            // relay: the leaf's average, a 32-bit float vector like every message
+  uint32_t fanin = 1;
+  std::vector<uint64_t> pulled_ts;   // fanin entries
 };
 
 struct OraclePS {
@@ -216,11 +251,14 @@ struct OraclePS {
   bool strict = false;             // fp32 evaluation, one fmaf per term (debugging aid)
   std::vector<float> theta, vel;   // vel: velocity (momentum SGD) or squared-gradient sum (AdaGrad)
   uint64_t ts = 0;
-  std::deque<Pending> fifo;
+  std::deque<Message> fifo;
+  uint64_t queued = 0;             // gradients the queued messages stand for
   // record of the most recent update
   std::vector<uint64_t> clock;     // vector clock <p_1..p_c> (Section 3.1)
   std::vector<uint32_t> sigma;
-  std::vector<float> scale;
+  std::vector<float> scale;        // per gradient: its message's step size over the message's fan-in
+  std::vector<float> msg_step;     // per message: the step size its vector is multiplied by
+  std::vector<uint32_t> msg_fanin;
   float abar = 0.f;
   double avg_sigma = 0.0;
 
@@ -236,55 +274,119 @@ struct OraclePS {
     return (double)f;
   }
 
+  double value_at(const Message& m, uint64_t k) const {
+    return m.fanin == 1 && m.avg.empty() ? grad_at(m.grad, k) : (double)m.avg[k];
+  }
+
   int64_t push(const void* g, uint64_t pulled_ts) {
     if (pulled_ts > ts) return -2;          // weights with that timestamp do not exist yet (Section 3.1)
-    fifo.push_back(Pending{g, pulled_ts});
-    return (int64_t)fifo.size();
+    Message m;
+    m.grad = g;
+    m.pulled_ts.assign(1, pulled_ts);
+    fifo.push_back(std::move(m));
+    queued += 1;
+    return (int64_t)queued;
+  }
+
+  // A leaf of the server tree (Section 3.3): averages the k gradients its learners sent, in
+  // arrival order, and relays the average to the root, which is this server.  Reading: the relay
+  // happens as soon as the leaf holds k gradients; the message carries all k timestamps, so the
+  // root's vector clock and Eq. 2 are those of a server that received the k gradients itself; a
+  // relayed average stands for k of the c gradients of an update and never straddles two updates.
+  int64_t push_relay(const void* const* g, const uint64_t* pulled, uint32_t k) {
+    if (k == 0 || k > c) return -1;
+    for (uint32_t l = 0; l < k; ++l)
+      if (pulled[l] > ts) return -2;
+    if (queued % c + k > c) return -5;
+    Message m;
+    m.fanin = k;
+    m.pulled_ts.assign(pulled, pulled + k);
+    m.avg.resize(N);
+    if (strict) {
+      const float inv_k = (float)(1.0 / (double)k);
+      for (uint64_t i = 0; i < N; ++i) {
+        float acc = 0.f;
+        for (uint32_t l = 0; l < k; ++l) acc = std::fmaf(inv_k, (float)grad_at(g[l], i), acc);
+        m.avg[i] = acc;
+      }
+    } else {
+      for (uint64_t i = 0; i < N; ++i) {
+        double sum = 0.0;
+        for (uint32_t l = 0; l < k; ++l) sum += grad_at(g[l], i);
+        m.avg[i] = (float)(sum / (double)k);   // the relayed message is a 32-bit float vector (Section 4.2)
+      }
+    }
+    fifo.push_back(std::move(m));
+    queued += k;
+    return (int64_t)queued;
   }
 
   int step() {
-    if (fifo.size() < c) return 0;
-    std::vector<Pending> grp(fifo.begin(), fifo.begin() + c);
+    if (queued < c) return 0;
+    // the leading messages that together stand for exactly c gradients
+    std::vector<Message> grp;
+    for (uint32_t have = 0; have < c;) {
+      have += fifo.front().fanin;
+      grp.push_back(std::move(fifo.front()));
+      fifo.pop_front();
+    }
+    queued -= c;
+    const uint32_t nmsg = (uint32_t)grp.size();
     // staleness of each gradient: server timestamp j minus gradient timestamp i (Section 3.1)
     clock.assign(c, 0);
     sigma.assign(c, 0);
+    std::vector<uint64_t> msg_sigma(nmsg, 0);   // sum of the staleness of the gradients a message stands for
     uint64_t sum_sigma = 0, sum_p = 0;
-    for (uint32_t l = 0; l < c; ++l) {
-      clock[l] = grp[l].pulled_ts;
-      sigma[l] = (uint32_t)(ts - grp[l].pulled_ts);
-      sum_sigma += sigma[l];
-      sum_p += grp[l].pulled_ts;
+    uint32_t l = 0;
+    for (uint32_t j = 0; j < nmsg; ++j) {
+      for (uint64_t p : grp[j].pulled_ts) {
+        clock[l] = p;
+        sigma[l] = (uint32_t)(ts - p);
+        msg_sigma[j] += sigma[l];
+        sum_sigma += sigma[l];
+        sum_p += p;
+        ++l;
+      }
     }
     // Eq. 2: <sigma> = (i-1) - mean(i_1..i_c), (i-1) being the timestamp before this update.
     avg_sigma = (double)ts - (double)sum_p / (double)c;
-    // Per-gradient step sizes: learning rate (Eq. 6, or a variant of it) times the 1/c of Eq. 5.
+    // Step size of each message: learning rate (Eq. 6, or a variant of it) times the share k/c of
+    // Eq. 5's average that the message stands for (k = 1 for a learner's own gradient: 1/c).
+    msg_step.assign(nmsg, 0.f);
+    msg_fanin.assign(nmsg, 0);
     scale.assign(c, 0.f);
     double sum_s = 0.0;
-    for (uint32_t l = 0; l < c; ++l) {
-      double div;
+    l = 0;
+    for (uint32_t j = 0; j < nmsg; ++j) {
+      const double k = (double)grp[j].fanin;
+      double num = (double)alpha0 * k, div;
       if (policy == LR_PAPER_N) {
         div = (double)n * (double)c;                                   // alpha0 / n, Eq. 6
       } else if (policy == LR_PER_GRADIENT) {
-        div = (double)std::max<uint32_t>(sigma[l], 1u) * (double)c;    // alpha0 / sigma_l (Section 5.1 footnote)
+        // alpha0 / sigma of the message (Section 5.1 footnote): the mean staleness of the gradients
+        // it stands for, floored at 1; alpha0 / max(sum/k, 1) = alpha0 k / max(sum, k)
+        num *= k;
+        div = (double)std::max<uint64_t>(msg_sigma[j], (uint64_t)grp[j].fanin) * (double)c;
       } else {
-        div = (double)std::max<uint64_t>(sum_sigma, (uint64_t)c);      // alpha0 / <sigma> of Eq. 2, then / c
+        div = (double)std::max<uint64_t>(sum_sigma, (uint64_t)c);      // alpha0 / <sigma> of Eq. 2, then k / c
       }
-      scale[l] = (float)((double)alpha0 / div);
-      sum_s += (double)scale[l];
+      msg_step[j] = (float)(num / div);
+      msg_fanin[j] = grp[j].fanin;
+      sum_s += (double)msg_step[j];
+      for (uint32_t i = 0; i < grp[j].fanin; ++i) scale[l++] = (float)((double)msg_step[j] / k);
     }
-    abar = (float)sum_s;   // the group's learning rate: sum of the per-gradient step sizes
+    abar = (float)sum_s;   // the group's learning rate: sum of the step sizes
 
     if (strict) {
       step_strict(grp);
       ts += 1;
-      fifo.erase(fifo.begin(), fifo.begin() + c);
       return 1;
     }
     for (uint64_t k = 0; k < N; ++k) {
       if (optimizer == OPT_MOMENTUM_SGD) {
         // sumGradients: staleness-scaled average of the c gradients (Eq. 5 with Eq. 6 folded in)
         double acc = 0.0;
-        for (uint32_t l = 0; l < c; ++l) acc += (double)scale[l] * grad_at(grp[l].grad, k);
+        for (uint32_t j = 0; j < nmsg; ++j) acc += (double)msg_step[j] * value_at(grp[j], k);
         // applyUpdate, reading: L2 penalty joins the gradient at the group's rate; heavy-ball
         // velocity carries the learning rate; with momentum = wd = 0 this is Eq. 5 exactly.
         double u = acc + (double)abar * (double)wd * (double)theta[k];
@@ -295,10 +397,10 @@ struct OraclePS {
       } else {
         // AdaGrad at the server (Section 5.5), reading: the averaged gradient of Eq. 5 plus the
         // L2 penalty feeds a running sum of squares; the step is rate * g / (sqrt(sum) + eps).
-        // (with a zero rate every step size is 0: the weights are then Eq. 5's plain 1/c)
+        // (with a zero rate every step size is 0: the weights are then Eq. 5's plain k/c)
         double gbar = 0.0;
-        for (uint32_t l = 0; l < c; ++l)
-          gbar += (abar > 0.f ? (double)scale[l] / (double)abar : 1.0 / (double)c) * grad_at(grp[l].grad, k);
+        for (uint32_t j = 0; j < nmsg; ++j)
+          gbar += (abar > 0.f ? (double)msg_step[j] / (double)abar : (double)grp[j].fanin / (double)c) * value_at(grp[j], k);
         gbar += (double)wd * (double)theta[k];
         double h = (double)vel[k] + gbar * gbar;
         double th = (double)theta[k] - (double)abar * gbar / (std::sqrt(h) + (double)adagrad_eps);
@@ -307,26 +409,26 @@ struct OraclePS {
       }
     }
     ts += 1;   // each weight update increments the timestamp by one (Section 3.1)
-    fifo.erase(fifo.begin(), fifo.begin() + c);
     return 1;
   }
 
-  // The same rule in fp32: acc = fma(s_l, g_l, acc) for l = 1..c from acc = 0, then one fma per
+  // The same rule in fp32: acc = fma(s_j, g_j, acc) over the messages from acc = 0, then one fma per
   // remaining term.  Same reading of momentum / decay / AdaGrad as above.
-  void step_strict(const std::vector<Pending>& grp) {
+  void step_strict(const std::vector<Message>& grp) {
     const float awd = (float)((double)abar * (double)wd);
+    const uint32_t nmsg = (uint32_t)grp.size();
     for (uint64_t k = 0; k < N; ++k) {
       float acc = 0.f;
       if (optimizer == OPT_MOMENTUM_SGD) {
-        for (uint32_t l = 0; l < c; ++l) acc = std::fmaf(scale[l], (float)grad_at(grp[l].grad, k), acc);
+        for (uint32_t j = 0; j < nmsg; ++j) acc = std::fmaf(msg_step[j], (float)value_at(grp[j], k), acc);
         const float u = std::fmaf(awd, theta[k], acc);
         const float v = momentum != 0.f ? std::fmaf(momentum, vel[k], u) : u;
         theta[k] = theta[k] - v;
         vel[k] = v;
       } else {
-        for (uint32_t l = 0; l < c; ++l) {
-          const float wl = abar > 0.f ? (float)((double)scale[l] / (double)abar) : (float)(1.0 / (double)c);
-          acc = std::fmaf(wl, (float)grad_at(grp[l].grad, k), acc);
+        for (uint32_t j = 0; j < nmsg; ++j) {
+          const float wj = abar > 0.f ? (float)((double)msg_step[j] / (double)abar) : (float)((double)grp[j].fanin / (double)c);
+          acc = std::fmaf(wj, (float)value_at(grp[j], k), acc);
         }
         const float g = std::fmaf(wd, theta[k], acc);
         const float h = std::fmaf(g, g, vel[k]);
@@ -353,11 +455,17 @@ void ora_splitmix64(uint64_t seed, uint64_t count, uint64_t* out) {
   for (uint64_t i = 0; i < count; ++i) out[i] = g.next();
 }
 
-void* ora_sched_create(uint32_t lambda, uint32_t n, int32_t mode, uint64_t seed, double ln_sigma, int32_t downcast) {
+void* ora_sched_create_tree(uint32_t lambda, uint32_t n, int32_t mode, uint64_t seed, double ln_sigma, int32_t downcast,
+                            uint32_t fanin) {
   if (lambda == 0 || n == 0 || n > lambda) return nullptr;
   if (mode < 0 || mode > 2) return nullptr;
   if (mode == MODE_HARDSYNC && n != 1) return nullptr;
-  return new OracleSched(lambda, n, mode, seed, ln_sigma, downcast != 0);
+  // a leaf's average stands for fanin of the c gradients of one update, and every learner has a leaf
+  if (fanin != 0 && (lambda % fanin != 0 || (lambda / n) % fanin != 0)) return nullptr;
+  return new OracleSched(lambda, n, mode, seed, ln_sigma, downcast != 0, fanin);
+}
+void* ora_sched_create(uint32_t lambda, uint32_t n, int32_t mode, uint64_t seed, double ln_sigma, int32_t downcast) {
+  return ora_sched_create_tree(lambda, n, mode, seed, ln_sigma, downcast, 0);
 }
 void ora_sched_destroy(void* s) { delete (OracleSched*)s; }
 // Writes count events into out (6 x 8-byte fields each: kind|learner packed as two 32-bit words,
@@ -385,8 +493,21 @@ void ora_ps_set_weights(void* p, const float* src) {
   for (uint64_t k = 0; k < P->N; ++k) { P->theta[k] = src[k]; P->vel[k] = 0.f; }
   P->ts = 0;
   P->fifo.clear();
+  P->queued = 0;
 }
 int64_t ora_ps_push(void* p, const void* grad, uint64_t pulled_ts) { return ((OraclePS*)p)->push(grad, pulled_ts); }
+int64_t ora_ps_push_relay(void* p, const void* const* grads, const uint64_t* pulled_ts, uint32_t k) {
+  return ((OraclePS*)p)->push_relay(grads, pulled_ts, k);
+}
+// Step sizes of the most recent update's messages and the number of gradients each stands for.
+int32_t ora_ps_last_messages(void* p, float* step, uint32_t* fanin) {
+  OraclePS* P = (OraclePS*)p;
+  for (size_t j = 0; j < P->msg_step.size(); ++j) {
+    if (step) step[j] = P->msg_step[j];
+    if (fanin) fanin[j] = P->msg_fanin[j];
+  }
+  return (int32_t)P->msg_step.size();
+}
 int32_t ora_ps_step(void* p) { return ((OraclePS*)p)->step(); }
 int64_t ora_ps_pull(void* p, float* dst) { return ((OraclePS*)p)->pull(dst); }
 int64_t ora_ps_timestamp(void* p) { return (int64_t)((OraclePS*)p)->ts; }

@@ -16,7 +16,7 @@ _SRC = os.path.join(_HERE, "rudra_oracle.cpp")
 _LIB = os.path.join(_HERE, "librudra_oracle.so")
 
 # event kinds / scheduler modes / options: integer values fixed by the event contract
-PUSH, STEP, PULL, PULL_SKIP, BROADCAST = 1, 2, 3, 4, 5
+PUSH, STEP, PULL, PULL_SKIP, BROADCAST, RELAY = 1, 2, 3, 4, 5, 6
 HARDSYNC, SOFTSYNC_ROUNDS, SOFTSYNC_TIMED = 0, 1, 2
 LR_PAPER_N, LR_PER_GRADIENT, LR_GROUP_MEAN = 0, 1, 2
 GRAD_F32, GRAD_BF16 = 0, 1
@@ -48,6 +48,8 @@ def lib():
         L.ora_splitmix64.argtypes = [C.c_uint64, C.c_uint64, C.c_void_p]
         L.ora_sched_create.restype = C.c_void_p
         L.ora_sched_create.argtypes = [C.c_uint32, C.c_uint32, C.c_int32, C.c_uint64, C.c_double, C.c_int32]
+        L.ora_sched_create_tree.restype = C.c_void_p
+        L.ora_sched_create_tree.argtypes = [C.c_uint32, C.c_uint32, C.c_int32, C.c_uint64, C.c_double, C.c_int32, C.c_uint32]
         L.ora_sched_destroy.argtypes = [C.c_void_p]
         L.ora_sched_run.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         L.ora_ps_create.restype = C.c_void_p
@@ -61,6 +63,10 @@ def lib():
         L.ora_ps_set_weights.argtypes = [C.c_void_p, C.c_void_p]
         L.ora_ps_push.restype = C.c_int64
         L.ora_ps_push.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
+        L.ora_ps_push_relay.restype = C.c_int64
+        L.ora_ps_push_relay.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32]
+        L.ora_ps_last_messages.restype = C.c_int32
+        L.ora_ps_last_messages.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.ora_ps_step.restype = C.c_int32
         L.ora_ps_step.argtypes = [C.c_void_p]
         L.ora_ps_pull.restype = C.c_int64
@@ -83,8 +89,9 @@ def splitmix64(seed, count):
 class OracleScheduler:
     """Event stream of lambda simulated learners (hardsync / n-softsync rounds / timed)."""
 
-    def __init__(self, lam, n, mode=SOFTSYNC_ROUNDS, seed=20150914, lognormal_sigma=0.3, downcast=False):
-        self._h = lib().ora_sched_create(lam, n, mode, seed, float(lognormal_sigma), int(bool(downcast)))
+    def __init__(self, lam, n, mode=SOFTSYNC_ROUNDS, seed=20150914, lognormal_sigma=0.3, downcast=False, fanin=0):
+        """fanin > 0: learners send to the leaves of a two-level server tree, fanin learners per leaf."""
+        self._h = lib().ora_sched_create_tree(lam, n, mode, seed, float(lognormal_sigma), int(bool(downcast)), int(fanin))
         if not self._h:
             raise ValueError("invalid scheduler arguments")
 
@@ -137,14 +144,36 @@ class OraclePS:
         want = np.float32 if self._dtype == GRAD_F32 else np.uint16
         g = np.ascontiguousarray(grad)
         assert g.dtype == want and g.size == self.N, (g.dtype, g.size)
-        self._keep.append(g)  # the oracle reads the buffer when the group closes
-        return lib().ora_ps_push(self._h, g.ctypes.data, int(pulled_ts))
+        r = lib().ora_ps_push(self._h, g.ctypes.data, int(pulled_ts))
+        if r > 0:
+            self._keep.append((1, g))  # the oracle reads the buffer when the group closes
+        return r
+
+    def push_relay(self, grads, pulled_ts):
+        """A leaf of the server tree averages ``grads`` (arrival order) and relays the average."""
+        want = np.float32 if self._dtype == GRAD_F32 else np.uint16
+        gs = [np.ascontiguousarray(g) for g in grads]
+        assert all(g.dtype == want and g.size == self.N for g in gs) and len(gs) == len(pulled_ts)
+        table = (C.c_void_p * len(gs))(*[g.ctypes.data for g in gs])
+        ts = np.ascontiguousarray(pulled_ts, dtype=np.uint64)
+        r = lib().ora_ps_push_relay(self._h, table, ts.ctypes.data, len(gs))
+        if r > 0:
+            self._keep.append((len(gs), None))  # averaged at once: the leaf does not keep the gradients
+        return r
 
     def step(self):
         r = lib().ora_ps_step(self._h)
         if r == 1:
-            del self._keep[: self.c]
+            have = 0
+            while have < self.c:
+                have += self._keep.pop(0)[0]
         return r
+
+    def last_messages(self):
+        step = np.zeros(self.c, dtype=np.float32)
+        fanin = np.zeros(self.c, dtype=np.uint32)
+        m = lib().ora_ps_last_messages(self._h, step.ctypes.data, fanin.ctypes.data)
+        return {"step": step[:m], "fanin": fanin[:m]}
 
     def pull(self):
         dst = np.empty(self.N, dtype=np.float32)
