@@ -65,6 +65,12 @@ typedef struct rudra_sched rudra_sched;
 #define RUDRA_OPT_OPTIMIZER 3
 #define   RUDRA_OPTIM_MOMENTUM_SGD 0 /* momentum-accelerated SGD with weight decay (Section 4.2) */
 #define   RUDRA_OPTIM_ADAGRAD      1 /* AdaGrad at the server (Section 5.5)                      */
+#define RUDRA_OPT_PUSH_MODE 4
+#define   RUDRA_PUSH_BORROW 0   /* a pushed device buffer is read by the update that consumes it */
+#define   RUDRA_PUSH_COPY   1   /* the server copies it at push time (Section 3.2: the message   */
+                                /* carries the gradient); costs one more read and write of it    */
+#define RUDRA_OPT_TREE_FANIN 5  /* learners per leaf when rudra_ps_run_events plays the server    */
+                                /* tree of Section 3.3; 0 (default): learners talk to the server */
 
 /*
  * rudra_ps_create -- a parameter server for a flat model of nparams weights, lambda learners and
@@ -107,6 +113,12 @@ int rudra_ps_set_weights_host(rudra_ps* ps, const float* src_host);
  */
 int64_t rudra_ps_push(rudra_ps* ps, const void* grad_dev, uint64_t pulled_ts);
 
+/* With RUDRA_OPT_PUSH_MODE = RUDRA_PUSH_COPY, rudra_ps_push (and the PUSH events of
+ * rudra_ps_run_events, and rudra_ps_push_group) copy the vector into a buffer the handle owns,
+ * on the handle's stream, before returning: the caller may overwrite or free grad_dev with any work
+ * ordered after the call on that stream.  For learners that cannot keep a buffer alive until the
+ * group closes.  Buffers are allocated on first use and re-used. */
+
 /* Same, for a gradient in host memory: it is copied into a staging buffer the handle owns
  * (allocated on first use, re-used afterwards) on an upload stream of the handle's own, so that
  * uploads, updates and rudra_ps_pull_host downloads overlap; the consuming update waits for the
@@ -125,6 +137,38 @@ int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_
  * gradients wait (nothing changes), < 0 on error.
  */
 int rudra_ps_step(rudra_ps* ps);
+
+/*
+ * The server tree of Section 3.3 (Rudra-adv), two levels.  A leaf node sits with the learners it is
+ * responsible for, averages the gradients they send and relays the average to its parent; the
+ * root -- this handle -- applies the update, and all weights keep one timestamp.
+ *
+ * rudra_leaf_average is the leaf's work: avg_dev[i] = mean over l of grads_dev[l][i] for k vectors
+ * of grad_dtype (RUDRA_GRAD_F32 / RUDRA_GRAD_BF16), nparams elements each; the result is a float
+ * vector like every message of the paper (Section 4.2).  It needs no handle and may run on the
+ * leaf's own GPU, with avg_dev in the root's memory (peer access enabled by the caller): k vectors
+ * are read locally and one crosses the link.  Per weight: k reads and one 4-byte write.
+ *
+ * rudra_ps_push_group hands the root one message that stands for k gradients, with the timestamps
+ * of all k (pulled_ts[0..k-1]): the root's vector clock, staleness and Eq. 2 are then those of a
+ * server that received the k gradients itself.  nvec == 1: vecs_dev[0] is the leaf's average (float;
+ * the handle's gradient type must be RUDRA_GRAD_F32).  nvec == k: vecs_dev[0..k-1] are the k raw
+ * gradients of the handle's gradient type, for a leaf that shares the root's GPU -- the update
+ * kernel averages them on the way and no intermediate vector is written.  The message takes the
+ * share k / c of Eq. 5's average at the rate of Eq. 6; under RUDRA_LR_PER_GRADIENT the rate is
+ * alpha0 / max(mean staleness of the message's gradients, 1).  A message must fit the open group
+ * (queued % c + k <= c, else RUDRA_E_STATE).  Buffers are borrowed or copied as in rudra_ps_push.
+ * Returns the number of gradients now queued.
+ *
+ * rudra_ps_last_messages reports, for the most recent update, how many gradients each of its
+ * messages stood for and the step size its vector was multiplied by; returns the message count.
+ * (rudra_ps_last_clock's scale_out is that step size divided by the fan-in, per gradient.)
+ */
+int rudra_leaf_average(const void* const* grads_dev, uint32_t k, int grad_dtype, uint64_t nparams, float* avg_dev,
+                       void* cuda_stream);
+int64_t rudra_ps_push_group(rudra_ps* ps, const void* const* vecs_dev, uint32_t nvec, const uint64_t* pulled_ts,
+                            uint32_t k);
+int rudra_ps_last_messages(const rudra_ps* ps, uint32_t* fanin_out, float* step_out);
 
 /* Like rudra_ps_step, and the same kernel also writes the new weights into k learner buffers
  * (dsts_dev: host array of k device pointers, each nparams floats, 0 <= k <= RUDRA_MAX_DSTS):
@@ -263,6 +307,7 @@ const char* rudra_noalloc_last_error(void);
 #define RUDRA_EV_PULL      3 /* learner receives the weights with timestamp ts                    */
 #define RUDRA_EV_PULL_SKIP 4 /* inquiry found the learner's copy current: no copy                 */
 #define RUDRA_EV_BROADCAST 5 /* all lambda learners receive the weights with timestamp ts         */
+#define RUDRA_EV_RELAY     6 /* server tree: leaf `learner` relays the average of its k gradients  */
 
 #define RUDRA_SCHED_HARDSYNC        0 /* Section 3.1 hardsync: n = 1, barrier, broadcast          */
 #define RUDRA_SCHED_SOFTSYNC_ROUNDS 1 /* every learner pushes once per round, seeded order        */
@@ -270,10 +315,11 @@ const char* rudra_noalloc_last_error(void);
 
 typedef struct rudra_event {
   int32_t  kind;       /* RUDRA_EV_*                                                            */
-  uint32_t learner;    /* learner the event belongs to (STEP: whose push closed the group)      */
+  uint32_t learner;    /* learner the event belongs to (STEP: whose push closed the group;     */
+                       /* RELAY: the leaf)                                                      */
   uint64_t pulled_ts;  /* PUSH: timestamp of the weights the gradient was computed from         */
   uint64_t ts;         /* PUSH: server timestamp at arrival; others: timestamp after the event  */
-  uint64_t seq;        /* PUSH: index of this learner's mini-batch, from 0                      */
+  uint64_t seq;        /* PUSH: index of this learner's mini-batch, from 0; RELAY: of the leaf's relay */
   uint64_t tick;       /* simulated arrival time (timed mode) or global push count (rounds)     */
 } rudra_event;
 
@@ -283,9 +329,21 @@ typedef struct rudra_event {
  * Returns NULL on invalid arguments. */
 rudra_sched* rudra_sched_create(uint32_t lambda, uint32_t n, int mode, uint64_t seed,
                                 double lognormal_sigma, int downcast);
+/* The same learners behind the two-level server tree of Section 3.3: learner l sends to leaf
+ * l / fanin; a leaf that holds fanin gradients relays their average to the root at once (a RELAY
+ * event right after the PUSH that filled it); the root updates when the averages it received stand
+ * for c gradients.  fanin must divide lambda and c = lambda / n; fanin = 0 is rudra_sched_create. */
+rudra_sched* rudra_sched_create_tree(uint32_t lambda, uint32_t n, int mode, uint64_t seed,
+                                     double lognormal_sigma, int downcast, uint32_t fanin);
 void rudra_sched_destroy(rudra_sched* s);
 /* Writes the next count events to out; returns count, or RUDRA_E_INVAL. */
 int64_t rudra_sched_next(rudra_sched* s, rudra_event* out, uint64_t count);
+/* For a caller that drives real learners: learner `learner` reports that the weights it now
+ * computes on carry timestamp ts (its pull was late, lost, or served from a cache), overriding
+ * what its last PULL / PULL_SKIP / BROADCAST event assumed.  Its next PUSH event then carries
+ * pulled_ts = ts.  Call it after reading that learner's pull event and before asking for further
+ * events.  RUDRA_E_BAD_TS if ts is ahead of the simulated server, RUDRA_E_INVAL for a bad learner. */
+int rudra_sched_on_pull(rudra_sched* s, uint32_t learner, uint64_t ts);
 
 /*
  * rudra_ps_run_events -- handle a backlog of messages.  Section 3.2's server takes messages one at
@@ -299,6 +357,10 @@ int64_t rudra_sched_next(rudra_sched* s, rudra_event* out, uint64_t count);
  * 32 updates, RUDRA_MAX_GROUP gradients and RUDRA_MAX_DSTS pull destinations per launch), every
  * gradient is read once and every pull is a store.  Per weight a window of W updates with P pulls
  * moves W*c*G + 16 + 4*P bytes instead of W*(c*G + 16) + 8*P.
+ *
+ * With RUDRA_OPT_TREE_FANIN = k the batch may come from rudra_sched_create_tree: PUSH events then
+ * deliver to the learner's leaf and each RELAY event hands the root that leaf's k gradients as one
+ * message (the leaves share this GPU: rudra_ps_push_group with nvec == k).
  *
  * grads_dev[l] is learner l's gradient buffer (read by the update that consumes the push, as in
  * rudra_ps_push), slots_dev[l] its weight buffer (written by its pulls and by broadcasts); both

@@ -468,6 +468,14 @@ void* ora_sched_create(uint32_t lambda, uint32_t n, int32_t mode, uint64_t seed,
   return ora_sched_create_tree(lambda, n, mode, seed, ln_sigma, downcast, 0);
 }
 void ora_sched_destroy(void* s) { delete (OracleSched*)s; }
+// A learner reports the timestamp of the weights it really computes on (a late or lost pull).
+int32_t ora_sched_on_pull(void* s, uint32_t learner, uint64_t ts) {
+  OracleSched* S = (OracleSched*)s;
+  if (learner >= S->lambda) return -1;
+  if (ts > S->ts) return -2;
+  S->local_ts[learner] = S->grad_ts[learner] = ts;
+  return 0;
+}
 // Writes count events into out (6 x 8-byte fields each: kind|learner packed as two 32-bit words,
 // pulled_ts, ts, seq, tick).
 void ora_sched_run(void* s, uint64_t count, Event* out) {

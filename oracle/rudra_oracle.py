@@ -51,6 +51,8 @@ def lib():
         L.ora_sched_create_tree.restype = C.c_void_p
         L.ora_sched_create_tree.argtypes = [C.c_uint32, C.c_uint32, C.c_int32, C.c_uint64, C.c_double, C.c_int32, C.c_uint32]
         L.ora_sched_destroy.argtypes = [C.c_void_p]
+        L.ora_sched_on_pull.restype = C.c_int32
+        L.ora_sched_on_pull.argtypes = [C.c_void_p, C.c_uint32, C.c_uint64]
         L.ora_sched_run.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         L.ora_ps_create.restype = C.c_void_p
         L.ora_ps_create.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_float, C.c_float, C.c_float]
@@ -99,6 +101,10 @@ class OracleScheduler:
         ev = np.zeros(count, dtype=EVENT_DTYPE)
         lib().ora_sched_run(self._h, count, ev.ctypes.data)
         return ev
+
+    def on_pull(self, learner, ts):
+        """The learner really computes on weights with timestamp ``ts`` (a late or lost pull)."""
+        return lib().ora_sched_on_pull(self._h, learner, ts)
 
     def __del__(self):
         if getattr(self, "_h", None):

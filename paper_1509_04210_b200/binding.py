@@ -16,11 +16,12 @@ from . import build as _build
 # constants of include/rudra_ps.h
 E_INVAL, E_BAD_TS, E_QUEUE_FULL, E_CUDA, E_STATE, E_NOMEM = -1, -2, -3, -4, -5, -6
 MAX_GROUP, MAX_DSTS, QUEUE_CAP, HIST_BINS = 128, 128, 4096, 4096
-OPT_GRAD_DTYPE, OPT_LR_POLICY, OPT_OPTIMIZER = 1, 2, 3
+OPT_GRAD_DTYPE, OPT_LR_POLICY, OPT_OPTIMIZER, OPT_PUSH_MODE, OPT_TREE_FANIN = 1, 2, 3, 4, 5
+PUSH_BORROW, PUSH_COPY = 0, 1
 GRAD_F32, GRAD_BF16 = 0, 1
 LR_PAPER_N, LR_PER_GRADIENT, LR_GROUP_MEAN = 0, 1, 2
 OPTIM_MOMENTUM_SGD, OPTIM_ADAGRAD = 0, 1
-EV_PUSH, EV_STEP, EV_PULL, EV_PULL_SKIP, EV_BROADCAST = 1, 2, 3, 4, 5
+EV_PUSH, EV_STEP, EV_PULL, EV_PULL_SKIP, EV_BROADCAST, EV_RELAY = 1, 2, 3, 4, 5, 6
 SCHED_HARDSYNC, SCHED_SOFTSYNC_ROUNDS, SCHED_SOFTSYNC_TIMED = 0, 1, 2
 
 EVENT_DTYPE = np.dtype(
@@ -65,6 +66,9 @@ def lib():
         "rudra_ps_set_weights_host": (C.c_int, [vp, vp]),
         "rudra_ps_push": (i64, [vp, vp, u64]),
         "rudra_ps_push_host": (i64, [vp, vp, u64]),
+        "rudra_ps_push_group": (i64, [vp, vp, u32, vp, u32]),
+        "rudra_ps_last_messages": (C.c_int, [vp, vp, vp]),
+        "rudra_leaf_average": (C.c_int, [vp, u32, C.c_int, u64, vp, vp]),
         "rudra_ps_step": (C.c_int, [vp]),
         "rudra_ps_step_pull_many": (C.c_int, [vp, vp, u32]),
         "rudra_ps_pull": (i64, [vp, vp]),
@@ -80,6 +84,8 @@ def lib():
         "rudra_ps_update_host_noalloc": (C.c_int, [vp, vp, u64, vp, vp, u32, f32, f32, vp]),
         "rudra_noalloc_last_error": (C.c_char_p, []),
         "rudra_sched_create": (vp, [u32, u32, C.c_int, u64, C.c_double, C.c_int]),
+        "rudra_sched_create_tree": (vp, [u32, u32, C.c_int, u64, C.c_double, C.c_int, u32]),
+        "rudra_sched_on_pull": (C.c_int, [vp, u32, u64]),
         "rudra_sched_destroy": (None, [vp]),
         "rudra_sched_next": (i64, [vp, vp, u64]),
         "rudra_ps_run_events": (i64, [vp, vp, u64, vp, vp, u32]),
@@ -147,13 +153,23 @@ def update_host_noalloc(theta_dev, state_dev, nparams, grads_host, scales, momen
     return code
 
 
+def leaf_average(grads_dev, grad_dtype, nparams, avg_dev, stream=None):
+    """rudra_leaf_average: what a leaf of the server tree does to the gradients of its learners."""
+    handle = stream.cuda_stream if hasattr(stream, "cuda_stream") else stream
+    return _check(lib().rudra_leaf_average(_ptr_array(grads_dev), len(grads_dev), int(grad_dtype), int(nparams),
+                                           _ptr(avg_dev), handle))
+
+
 class Scheduler:
     """rudra_sched_*: the arrival order of push / pull messages of lambda simulated learners."""
 
-    def __init__(self, lam, n, mode=SCHED_SOFTSYNC_ROUNDS, seed=20150914, lognormal_sigma=0.3, downcast=False):
-        self._h = lib().rudra_sched_create(lam, n, mode, seed, float(lognormal_sigma), int(bool(downcast)))
+    def __init__(self, lam, n, mode=SCHED_SOFTSYNC_ROUNDS, seed=20150914, lognormal_sigma=0.3, downcast=False, fanin=0):
+        self._h = lib().rudra_sched_create_tree(lam, n, mode, seed, float(lognormal_sigma), int(bool(downcast)), int(fanin))
         if not self._h:
             raise ValueError("invalid scheduler arguments")
+
+    def on_pull(self, learner, ts):
+        return _check(lib().rudra_sched_on_pull(self._h, int(learner), int(ts)))
 
     def next(self, count):
         ev = np.zeros(count, dtype=EVENT_DTYPE)
@@ -206,6 +222,17 @@ class ParameterServer:
 
     def push_host(self, grad_host, pulled_ts):
         return _check(lib().rudra_ps_push_host(self._h, _ptr(grad_host), int(pulled_ts)))
+
+    def push_group(self, vecs_dev, pulled_ts):
+        """One message standing for len(pulled_ts) gradients: their average (one vector) or the raw vectors."""
+        ts = np.ascontiguousarray(pulled_ts, dtype=np.uint64)
+        return _check(lib().rudra_ps_push_group(self._h, _ptr_array(vecs_dev), len(vecs_dev), ts.ctypes.data, len(ts)))
+
+    def last_messages(self):
+        fanin = np.zeros(MAX_GROUP, dtype=np.uint32)
+        step = np.zeros(MAX_GROUP, dtype=np.float32)
+        m = _check(lib().rudra_ps_last_messages(self._h, fanin.ctypes.data, step.ctypes.data))
+        return {"fanin": fanin[:m], "step": step[:m]}
 
     def step(self):
         return _check(lib().rudra_ps_step(self._h))

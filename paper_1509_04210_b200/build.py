@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_PKG, "librudra_ps.so")
-SOURCES = ["ps.cu", "update.cu", "snapshot.cu", "noalloc.cu", "sched.cpp"]
+SOURCES = ["ps.cu", "update.cu", "snapshot.cu", "leaf.cu", "noalloc.cu", "sched.cpp"]
 # measurement utility of the benchmark, a library of its own: not part of the product interface
 PROBE_LIB_PATH = os.path.join(_PKG, "librudra_probe.so")
 PROBE_SOURCES = ["probe.cu"]

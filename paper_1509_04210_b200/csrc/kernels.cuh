@@ -17,20 +17,22 @@ constexpr int kMaxWindow = 32;   // most updates one launch can carry
 // sumGradients + applyUpdate over c gradients) with the pulls that fall between them.  Passed by
 // value as a __grid_constant__ kernel parameter: the gradient pointers, step sizes and pull
 // destinations form a small table in the constant bank, read with uniform addresses, so a window
-// costs one launch and no other stream operation.  Update u uses grad[u*c .. u*c+c-1]; pull
-// destinations dst[dst_end[u] .. dst_end[u+1]-1] receive the weights after update u, and
-// dst[0 .. dst_end[0]-1] the weights as they were before the window.
+// costs one launch and no other stream operation.  Update u uses the vectors
+// grad[grad_end[u] .. grad_end[u+1]-1] (c of them when every learner's gradient arrives by itself,
+// fewer when leaves of a server tree relay averages); pull destinations
+// dst[dst_end[u] .. dst_end[u+1]-1] receive the weights after update u, and dst[0 .. dst_end[0]-1]
+// the weights as they were before the window.
 struct UpdateParams {
-  const void* grad[kMaxGroup];   // nupd * c gradient vectors, arrival order
+  const void* grad[kMaxGroup];   // the window's gradient vectors, arrival order
   float* dst[kMaxDsts];          // learner buffers, in the order the pulls arrived
-  float scale[kMaxGroup];        // s_l (momentum SGD) or s_l / sum(s) (AdaGrad), aligned with grad[]
+  float scale[kMaxGroup];        // step size (momentum SGD) or weight in the mean (AdaGrad), aligned with grad[]
   float awd[kMaxWindow];         // per update, momentum SGD: sum(s) * weight_decay
   float abar[kMaxWindow];        // per update, AdaGrad: sum(s), the group's learning rate
   uint8_t dst_end[kMaxWindow + 1];
+  uint8_t grad_end[kMaxWindow + 2];   // grad_end[0] = 0; one spare entry, read but never used, after the last update
   float* theta;
   float* state;                  // velocity (momentum SGD) or sum of squared gradients (AdaGrad)
   uint64_t n;                    // number of weights
-  uint32_t c;                    // gradients per update
   uint32_t nupd;                 // updates in this window (>= 1)
   float momentum;
   float wd;                      // AdaGrad: weight decay
@@ -54,5 +56,15 @@ cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, in
 
 // Enqueue one 1 -> ndst copy of the weights.
 cudaError_t launch_snapshot(const SnapshotParams& p, cudaStream_t stream);
+
+// What a leaf of the server tree does (Section 3.3): out[i] = mean of k gradient vectors at i.
+struct LeafParams {
+  const void* grad[kMaxGroup];
+  float* out;
+  uint64_t n;
+  uint32_t k;
+  float inv_k;
+};
+cudaError_t launch_leaf_average(const LeafParams& p, GradType gtype, cudaStream_t stream);
 
 }  // namespace rudra

@@ -103,8 +103,9 @@ int rudra_ps_update_host_noalloc(float* theta_dev, float* state_dev, uint64_t np
   p.theta = theta_dev;
   p.state = state_dev;
   p.n = nparams;
-  p.c = c;
   p.nupd = 1;
+  p.grad_end[0] = 0;
+  p.grad_end[1] = p.grad_end[2] = (uint8_t)c;
   p.dst_end[0] = p.dst_end[1] = 0;
   p.momentum = momentum;
   p.awd[0] = (float)((double)abar * (double)weight_decay);

@@ -52,10 +52,17 @@ constexpr uintptr_t kAlignMask = 31;       // 256-bit vector accesses
 
 bool aligned(const void* p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & kAlignMask) == 0; }
 
+// One gradient the queue stands for.  A learner's own gradient is a message of one entry.  The
+// average a leaf of the server tree relays for k gradients (Section 3.3) is a message of k entries,
+// one per timestamp it carries: the first holds the vector (the leaf's average), the others none.
+// A leaf that shares the server's GPU hands over its k raw vectors instead, one per entry, and the
+// update kernel does the averaging.
 struct Pending {
-  const void* grad;
+  const void* grad;     // vector to read, or nullptr (an entry of an averaged message after the first)
   uint64_t pulled_ts;
-  int slot;   // staging slot that holds the data, or -1 for a borrowed caller buffer
+  int slot;             // staging slot that holds the data, or -1 for a borrowed caller buffer
+  uint32_t fanin;       // first entry of a message: gradients it stands for; later entries: 0
+  bool uploaded;        // the slot is filled by the upload stream: its reader waits for slot_ready
 };
 
 // Makes the handle's device current for the duration of a call.
@@ -81,6 +88,9 @@ struct rudra_ps {
   uint32_t lambda = 0, n = 0, c = 0;
   float alpha0 = 0.f, momentum = 0.f, wd = 0.f, eps = 1e-8f;
   int gtype = RUDRA_GRAD_F32, policy = RUDRA_LR_PAPER_N, optim = RUDRA_OPTIM_MOMENTUM_SGD;
+  int push_mode = RUDRA_PUSH_BORROW;
+  uint32_t fanin = 0;              // learners per leaf when rudra_ps_run_events plays a server tree; 0 = none
+  std::vector<std::vector<Pending>> leaf_pending;   // per leaf: gradients received, not yet relayed
   int device = 0;
   int sm_count = 0;
   uint32_t sweep = 0;              // launches so far: successive launches sweep in opposite directions
@@ -104,6 +114,8 @@ struct rudra_ps {
   std::vector<uint64_t> clock;
   std::vector<uint32_t> sigma;
   std::vector<float> scale;
+  std::vector<float> msg_step;     // last update: step size of each message
+  std::vector<uint32_t> msg_fanin; // last update: gradients each message stood for
   double avg_sigma = 0.0;
   // Record of past updates (Section 3.2: the server records the vector clock of each weight
   // update to keep track of the average staleness): a ring of the last kClockLog updates, c
@@ -134,6 +146,11 @@ void release_queue(rudra_ps* ps) {
   for (const Pending& e : ps->queue)
     if (e.slot >= 0) ps->free_slots.push_back(e.slot);
   ps->queue.clear();
+  for (auto& leaf : ps->leaf_pending) {
+    for (const Pending& e : leaf)
+      if (e.slot >= 0) ps->free_slots.push_back(e.slot);
+    leaf.clear();
+  }
 }
 
 cudaError_t sync_all(rudra_ps* ps) {
@@ -176,10 +193,53 @@ void free_host_path(rudra_ps* ps) {
   ps->up_stream = ps->down_stream = nullptr;
 }
 
-int64_t enqueue(rudra_ps* ps, const void* grad, uint64_t pulled_ts, int slot) {
-  ps->queue.push_back(Pending{grad, pulled_ts, slot});
+int64_t enqueue(rudra_ps* ps, const void* grad, uint64_t pulled_ts, int slot, bool uploaded = false) {
+  ps->queue.push_back(Pending{grad, pulled_ts, slot, 1u, uploaded});
   ps->counters[0] += 1;
   return (int64_t)ps->queue.size();
+}
+
+// A staging slot of grad_bytes() bytes: a free one, else a new allocation.  *fresh tells whether it
+// was just allocated (no earlier reader to wait for).
+cudaError_t acquire_slot(rudra_ps* ps, int* slot, bool* fresh) {
+  if (!ps->free_slots.empty()) {
+    *slot = ps->free_slots.back();
+    ps->free_slots.pop_back();
+    *fresh = false;
+    return cudaSuccess;
+  }
+  void* buf = nullptr;
+  cudaEvent_t ready = nullptr, spent = nullptr;
+  cudaError_t e = cudaMalloc(&buf, ps->grad_bytes());
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ready, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&spent, cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    cudaFree(buf);
+    if (ready) cudaEventDestroy(ready);
+    return e;
+  }
+  ps->slots.push_back(buf);
+  ps->slot_ready.push_back(ready);
+  ps->slot_spent.push_back(spent);
+  *slot = (int)ps->slots.size() - 1;
+  *fresh = true;
+  return cudaSuccess;
+}
+
+// COPY push mode (Section 3.2: the push message carries the gradient itself): the vector is copied
+// into a staging slot on the handle's stream at push time, so the caller's buffer is free again
+// for anything ordered after this call on that stream.  The slot's last reader ran on the same
+// stream, so the copy needs no event.
+int stage_device_copy(rudra_ps* ps, const void* src, int* slot) {
+  bool fresh = false;
+  cudaError_t e = acquire_slot(ps, slot, &fresh);
+  if (e != cudaSuccess) return cuda_fail(e, "staging buffer allocation");
+  e = cudaMemcpyAsync(ps->slots[*slot], src, ps->grad_bytes(), cudaMemcpyDeviceToDevice, ps->stream);
+  if (e != cudaSuccess) {
+    ps->free_slots.push_back(*slot);
+    return cuda_fail(e, "gradient device-to-device copy");
+  }
+  return 0;
 }
 
 int check_push(rudra_ps* ps, uint64_t pulled_ts) {
@@ -238,16 +298,28 @@ struct ViewBook {
   }
 };
 
-// Group close (Section 3.1, Eq. 2) and the step-size table (Eq. 5's 1/c times the rate of Eq. 6
-// or one of its two variants) for the c oldest queued gradients, appended to the window as its
-// next update.  Integers first, then one rounding to fp32 per table entry.  Raises the timestamp.
+// Vectors the next update will read: one per learner's own gradient, one per relayed average, k per
+// group of raw vectors handed over by a leaf on this GPU.
+uint32_t next_update_vectors(const rudra_ps* ps) {
+  uint32_t nvec = 0;
+  for (uint32_t l = 0; l < ps->c; ++l) nvec += ps->queue[l].grad != nullptr;
+  return nvec;
+}
+
+// Group close (Section 3.1, Eq. 2) and the step-size table (Eq. 5's share of the average times the
+// rate of Eq. 6 or one of its two variants) for the messages that stand for the c oldest queued
+// gradients, appended to the window as its next update.  Integers first, then one rounding to
+// fp32 per table entry.  Raises the timestamp.
 void append_update(rudra_ps* ps, Window& w) {
   const uint32_t c = ps->c;
   rudra::UpdateParams& p = w.p;
-  const uint32_t base = w.nupd * c;
+  if (w.nupd == 0) p.grad_end[0] = 0;
+  uint32_t vec = p.grad_end[w.nupd];
   ps->clock.resize(c);
   ps->sigma.resize(c);
   ps->scale.resize(c);
+  ps->msg_step.clear();
+  ps->msg_fanin.clear();
   uint64_t sum_sigma = 0, sum_pulled = 0;
   for (uint32_t l = 0; l < c; ++l) {
     const Pending& e = ps->queue[l];
@@ -255,10 +327,11 @@ void append_update(rudra_ps* ps, Window& w) {
     ps->sigma[l] = (uint32_t)(ps->ts - e.pulled_ts);
     sum_sigma += ps->sigma[l];
     sum_pulled += e.pulled_ts;
-    p.grad[base + l] = e.grad;
     if (e.slot >= 0) {
-      const cudaError_t we = cudaStreamWaitEvent(ps->stream, ps->slot_ready[e.slot], 0);   // the kernel starts after its uploads
-      if (we != cudaSuccess && w.wait_error == cudaSuccess) w.wait_error = we;
+      if (e.uploaded) {   // the kernel starts after its uploads
+        const cudaError_t we = cudaStreamWaitEvent(ps->stream, ps->slot_ready[e.slot], 0);
+        if (we != cudaSuccess && w.wait_error == cudaSuccess) w.wait_error = we;
+      }
       w.used_slots.push_back(e.slot);
     }
   }
@@ -279,35 +352,67 @@ void append_update(rudra_ps* ps, Window& w) {
       ps->sigma_hist[bin] += 1;
     }
   }
-  double sum_scale = 0.0;
-  for (uint32_t l = 0; l < c; ++l) {
-    double divisor;
+  // Step size of each message: rate times the share k / c of Eq. 5's average it stands for.
+  double sum_step = 0.0;
+  for (uint32_t l = 0; l < c;) {
+    const uint32_t k = ps->queue[l].fanin;
+    uint64_t msg_sigma = 0;
+    for (uint32_t i = 0; i < k; ++i) msg_sigma += ps->sigma[l + i];
+    double num = (double)ps->alpha0 * (double)k, divisor;
     switch (ps->policy) {
-      case RUDRA_LR_PER_GRADIENT: divisor = (double)(ps->sigma[l] > 1 ? ps->sigma[l] : 1u) * (double)c; break;
-      case RUDRA_LR_GROUP_MEAN:   divisor = (double)(sum_sigma > c ? sum_sigma : (uint64_t)c); break;
-      default:                    divisor = (double)ps->n * (double)c; break;
+      case RUDRA_LR_PER_GRADIENT:   // alpha0 / max(mean staleness of the message, 1) = alpha0 k / max(sum, k)
+        num *= (double)k;
+        divisor = (double)(msg_sigma > k ? msg_sigma : (uint64_t)k) * (double)c;
+        break;
+      case RUDRA_LR_GROUP_MEAN:     // alpha0 / max(<sigma>, 1) with Eq. 2's <sigma> = sum / c
+        divisor = (double)(sum_sigma > c ? sum_sigma : (uint64_t)c);
+        break;
+      default:                      // alpha0 / n
+        divisor = (double)ps->n * (double)c;
+        break;
     }
-    ps->scale[l] = (float)((double)ps->alpha0 / divisor);
-    sum_scale += (double)ps->scale[l];
+    const float step = (float)(num / divisor);
+    ps->msg_step.push_back(step);
+    ps->msg_fanin.push_back(k);
+    sum_step += (double)step;
+    for (uint32_t i = 0; i < k; ++i) ps->scale[l + i] = (float)((double)step / (double)k);
+    l += k;
   }
-  const float abar = (float)sum_scale;
-  for (uint32_t l = 0; l < c; ++l) {
-    // AdaGrad combines the gradients with weights s_l / sum(s); with a zero rate every s_l is 0 and
-    // the weights fall back to Eq. 5's plain 1/c (the weights do not move, the sum of squares does)
-    const float weight = abar > 0.f ? (float)((double)ps->scale[l] / (double)abar) : (float)(1.0 / (double)c);
-    p.scale[base + l] = ps->optim == RUDRA_OPTIM_ADAGRAD ? weight : ps->scale[l];
+  const float abar = (float)sum_step;
+  // The kernel's table: one entry per vector.  An averaged message is one vector with the
+  // message's step size; raw vectors get their message's step size over its fan-in each.
+  // AdaGrad combines the vectors with weights (step / sum of steps); with a zero rate every step
+  // is 0 and the weights fall back to Eq. 5's plain shares (the weights do not move, the sum of
+  // squares does).
+  uint32_t m = 0;
+  for (uint32_t l = 0; l < c; ++m) {
+    const uint32_t k = ps->queue[l].fanin;
+    uint32_t nvec = 0;
+    for (uint32_t i = 0; i < k; ++i) nvec += ps->queue[l + i].grad != nullptr;
+    const double step = (double)ps->msg_step[m];
+    const double weight = abar > 0.f ? step / (double)abar : (double)k / (double)c;
+    for (uint32_t i = 0; i < k; ++i) {
+      const Pending& e = ps->queue[l + i];
+      if (!e.grad) continue;
+      p.grad[vec] = e.grad;
+      p.scale[vec] = (float)((ps->optim == RUDRA_OPTIM_ADAGRAD ? weight : step) / (double)nvec);
+      vec += 1;
+    }
+    l += k;
   }
   p.awd[w.nupd] = (float)((double)abar * (double)ps->wd);
   p.abar[w.nupd] = abar;
   p.dst_end[w.nupd] = (uint8_t)w.ndst;   // pulls so far belong to the state before this update
   w.nupd += 1;
+  p.grad_end[w.nupd] = (uint8_t)vec;
   ps->has_clock = true;
   for (uint32_t l = 0; l < c; ++l) ps->queue.pop_front();
   ps->ts += 1;   // exactly one increment per weight update
 }
 
 bool window_has_room_for_update(const rudra_ps* ps, const Window& w, uint32_t max_updates) {
-  return w.nupd < max_updates && (w.nupd + 1) * ps->c <= (uint32_t)rudra::kMaxGroup;
+  const uint32_t used = w.nupd ? w.p.grad_end[w.nupd] : 0;
+  return w.nupd < max_updates && used + next_update_vectors(ps) <= (uint32_t)rudra::kMaxGroup;
 }
 
 // Enqueues the window: the fused kernel if it holds updates, a plain snapshot if it holds only pulls.
@@ -348,8 +453,8 @@ int flush_window(rudra_ps* ps, Window& w) {
     p.theta = ps->theta;
     p.state = ps->state;
     p.n = ps->N;
-    p.c = ps->c;
     p.nupd = w.nupd;
+    p.grad_end[w.nupd + 1] = p.grad_end[w.nupd];
     p.momentum = ps->momentum;
     p.wd = ps->wd;
     p.eps = ps->eps;
@@ -484,6 +589,18 @@ int rudra_ps_set_option(rudra_ps* ps, int key, int64_t value) {
           ps->optim = (int)value;
         }
         return 0;
+      case RUDRA_OPT_PUSH_MODE:
+        if (value != RUDRA_PUSH_BORROW && value != RUDRA_PUSH_COPY) return fail(RUDRA_E_INVAL, "unknown push mode %lld", (long long)value);
+        ps->push_mode = (int)value;
+        return 0;
+      case RUDRA_OPT_TREE_FANIN:
+        if (value < 0 || (value > 0 && (ps->lambda % value != 0 || ps->c % value != 0)))
+          return fail(RUDRA_E_INVAL, "fan-in %lld must divide lambda = %u and c = %u", (long long)value, ps->lambda, ps->c);
+        for (const auto& leaf : ps->leaf_pending)
+          if (!leaf.empty()) return fail(RUDRA_E_STATE, "leaves still hold gradients");
+        ps->fanin = (uint32_t)value;
+        ps->leaf_pending.assign(value ? ps->lambda / (uint32_t)value : 0, {});
+        return 0;
       default:
         return fail(RUDRA_E_INVAL, "unknown option key %d", key);
     }
@@ -528,7 +645,11 @@ int64_t rudra_ps_push(rudra_ps* ps, const void* grad_dev, uint64_t pulled_ts) {
     if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
     if (!aligned(grad_dev)) return fail(RUDRA_E_INVAL, "gradient pointer is null or not 32-byte aligned");
     if (int r = check_push(ps, pulled_ts)) return r;
-    return enqueue(ps, grad_dev, pulled_ts, -1);
+    if (ps->push_mode == RUDRA_PUSH_BORROW) return enqueue(ps, grad_dev, pulled_ts, -1);
+    DeviceScope dev(ps->device);
+    int slot = -1;
+    if (int r = stage_device_copy(ps, grad_dev, &slot)) return r;
+    return enqueue(ps, ps->slots[slot], pulled_ts, slot);
   });
 }
 
@@ -540,30 +661,18 @@ int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_
     DeviceScope dev(ps->device);
     cudaError_t e = ensure_copy_streams(ps);
     if (e != cudaSuccess) return cuda_fail(e, "copy stream creation");
-    int slot;
-    if (!ps->free_slots.empty()) {
-      slot = ps->free_slots.back();
-      ps->free_slots.pop_back();
-      e = cudaStreamWaitEvent(ps->up_stream, ps->slot_spent[slot], 0);   // its last reader must be done
+    int slot = -1;
+    bool fresh = false;
+    e = acquire_slot(ps, &slot, &fresh);
+    if (e != cudaSuccess) return cuda_fail(e, "staging buffer allocation");
+    if (!fresh) {
+      // the slot's last reader must be done; a slot last filled by a COPY-mode push was read on the
+      // main stream too, and its slot_spent was recorded after that launch
+      e = cudaStreamWaitEvent(ps->up_stream, ps->slot_spent[slot], 0);
       if (e != cudaSuccess) {
         ps->free_slots.push_back(slot);
         return cuda_fail(e, "cudaStreamWaitEvent");
       }
-    } else {
-      void* buf = nullptr;
-      cudaEvent_t ready = nullptr, spent = nullptr;
-      e = cudaMalloc(&buf, ps->grad_bytes());
-      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ready, cudaEventDisableTiming);
-      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&spent, cudaEventDisableTiming);
-      if (e != cudaSuccess) {
-        cudaFree(buf);
-        if (ready) cudaEventDestroy(ready);
-        return cuda_fail(e, "staging buffer allocation");
-      }
-      ps->slots.push_back(buf);
-      ps->slot_ready.push_back(ready);
-      ps->slot_spent.push_back(spent);
-      slot = (int)ps->slots.size() - 1;
     }
     e = cudaMemcpyAsync(ps->slots[slot], grad_host, ps->grad_bytes(), cudaMemcpyHostToDevice, ps->up_stream);
     if (e == cudaSuccess) e = cudaEventRecord(ps->slot_ready[slot], ps->up_stream);
@@ -572,7 +681,90 @@ int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_
       return cuda_fail(e, "gradient host-to-device copy");
     }
     ps->counters[4] += ps->grad_bytes();
-    return enqueue(ps, ps->slots[slot], pulled_ts, slot);
+    return enqueue(ps, ps->slots[slot], pulled_ts, slot, true);
+  });
+}
+
+// Appends one message that stands for k gradients: vecs[0..nvec-1] with nvec == 1 (an average) or
+// nvec == k (raw vectors).  Arguments are already validated.
+static int64_t enqueue_group(rudra_ps* ps, const Pending* vecs, uint32_t nvec, const uint64_t* pulled_ts, uint32_t k) {
+  for (uint32_t i = 0; i < k; ++i) {
+    Pending e = i < nvec ? vecs[i] : Pending{nullptr, 0, -1, 0u, false};
+    e.pulled_ts = pulled_ts[i];
+    e.fanin = i == 0 ? k : 0u;
+    ps->queue.push_back(e);
+  }
+  ps->counters[0] += k;
+  return (int64_t)ps->queue.size();
+}
+
+int64_t rudra_ps_push_group(rudra_ps* ps, const void* const* vecs_dev, uint32_t nvec, const uint64_t* pulled_ts,
+                            uint32_t k) {
+  return guarded([&]() -> int64_t {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (k == 0 || k > ps->c || !vecs_dev || !pulled_ts) return fail(RUDRA_E_INVAL, "need 1 <= k <= c and non-null tables");
+    if (nvec != 1 && nvec != k) return fail(RUDRA_E_INVAL, "nvec must be 1 (an average) or k (raw gradients)");
+    if (nvec == 1 && k > 1 && ps->gtype != RUDRA_GRAD_F32)
+      return fail(RUDRA_E_STATE, "a relayed average is a float vector: the handle's gradient type must be RUDRA_GRAD_F32");
+    for (uint32_t i = 0; i < nvec; ++i)
+      if (!aligned(vecs_dev[i])) return fail(RUDRA_E_INVAL, "vector %u is null or not 32-byte aligned", i);
+    for (uint32_t i = 0; i < k; ++i)
+      if (pulled_ts[i] > ps->ts)
+        return fail(RUDRA_E_BAD_TS, "pulled_ts[%u] = %llu is ahead of the server timestamp %llu", i,
+                    (unsigned long long)pulled_ts[i], (unsigned long long)ps->ts);
+    if (ps->queue.size() % ps->c + k > ps->c)
+      return fail(RUDRA_E_STATE, "a message for %u gradients does not fit the open group (%zu of %u queued)", k,
+                  ps->queue.size() % ps->c, ps->c);
+    if (ps->queue.size() + k > RUDRA_QUEUE_CAP) return fail(RUDRA_E_QUEUE_FULL, "%d gradients already queued", RUDRA_QUEUE_CAP);
+    Pending vecs[RUDRA_MAX_GROUP];
+    DeviceScope dev(ps->device);
+    for (uint32_t i = 0; i < nvec; ++i) {
+      vecs[i] = Pending{vecs_dev[i], 0, -1, 0u, false};
+      if (ps->push_mode == RUDRA_PUSH_COPY) {
+        int slot = -1;
+        if (int r = stage_device_copy(ps, vecs_dev[i], &slot)) {
+          for (uint32_t u = 0; u < i; ++u) ps->free_slots.push_back(vecs[u].slot);
+          return r;
+        }
+        vecs[i].grad = ps->slots[slot];
+        vecs[i].slot = slot;
+      }
+    }
+    return enqueue_group(ps, vecs, nvec, pulled_ts, k);
+  });
+}
+
+int rudra_ps_last_messages(const rudra_ps* ps, uint32_t* fanin_out, float* step_out) {
+  return guarded([&]() -> int {
+    if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
+    if (!ps->has_clock) return 0;
+    for (size_t j = 0; j < ps->msg_step.size(); ++j) {
+      if (fanin_out) fanin_out[j] = ps->msg_fanin[j];
+      if (step_out) step_out[j] = ps->msg_step[j];
+    }
+    return (int)ps->msg_step.size();
+  });
+}
+
+int rudra_leaf_average(const void* const* grads_dev, uint32_t k, int grad_dtype, uint64_t nparams, float* avg_dev,
+                       void* cuda_stream) {
+  return guarded([&]() -> int {
+    if (k == 0 || k > RUDRA_MAX_GROUP || !grads_dev || nparams == 0) return fail(RUDRA_E_INVAL, "need 1 <= k <= RUDRA_MAX_GROUP, nparams > 0 and a gradient table");
+    if (grad_dtype != RUDRA_GRAD_F32 && grad_dtype != RUDRA_GRAD_BF16) return fail(RUDRA_E_INVAL, "unknown gradient type %d", grad_dtype);
+    if (!aligned(avg_dev)) return fail(RUDRA_E_INVAL, "output is null or not 32-byte aligned");
+    rudra::LeafParams p;
+    for (uint32_t l = 0; l < k; ++l) {
+      if (!aligned(grads_dev[l])) return fail(RUDRA_E_INVAL, "gradient %u is null or not 32-byte aligned", l);
+      p.grad[l] = grads_dev[l];
+    }
+    p.out = avg_dev;
+    p.n = nparams;
+    p.k = k;
+    p.inv_k = (float)(1.0 / (double)k);
+    const cudaError_t e = rudra::launch_leaf_average(p, grad_dtype == RUDRA_GRAD_BF16 ? rudra::kBF16 : rudra::kF32,
+                                                     static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "leaf average kernel launch");
+    return 0;
   });
 }
 
@@ -597,6 +789,9 @@ int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t co
       uint64_t queued = ps->queue.size();
       ViewBook sim(ps);
       bool fresh;
+      const uint32_t fanin = ps->fanin;
+      std::vector<uint32_t> leaf_fill(ps->leaf_pending.size());
+      for (size_t j = 0; j < leaf_fill.size(); ++j) leaf_fill[j] = (uint32_t)ps->leaf_pending[j].size();
       for (uint64_t i = 0; i < count; ++i) {
         const rudra_event& ev = events[i];
         const bool needs_learner = ev.kind == RUDRA_EV_PUSH || ev.kind == RUDRA_EV_PULL;
@@ -606,7 +801,20 @@ int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t co
             if (!grads_dev || !aligned(grads_dev[ev.learner])) return fail(RUDRA_E_INVAL, "event %llu: gradient buffer of learner %u is null or not 32-byte aligned", (unsigned long long)i, ev.learner);
             if (ev.pulled_ts > ts) return fail(RUDRA_E_BAD_TS, "event %llu: pulled_ts %llu is ahead of the server timestamp %llu", (unsigned long long)i, (unsigned long long)ev.pulled_ts, (unsigned long long)ts);
             if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: push expects server timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+            if (fanin) {   // the gradient goes to the learner's leaf, not to the root's queue
+              if (++leaf_fill[ev.learner / fanin] > fanin) return fail(RUDRA_E_STATE, "event %llu: leaf %u holds more than %u gradients without a relay", (unsigned long long)i, ev.learner / fanin, fanin);
+              break;
+            }
             if (++queued > RUDRA_QUEUE_CAP) return fail(RUDRA_E_QUEUE_FULL, "event %llu: queue full", (unsigned long long)i);
+            break;
+          case RUDRA_EV_RELAY:
+            if (!fanin) return fail(RUDRA_E_STATE, "event %llu: relay, but RUDRA_OPT_TREE_FANIN is not set", (unsigned long long)i);
+            if (ev.learner >= leaf_fill.size()) return fail(RUDRA_E_INVAL, "event %llu: leaf %u out of range", (unsigned long long)i, ev.learner);
+            if (leaf_fill[ev.learner] != fanin) return fail(RUDRA_E_STATE, "event %llu: leaf %u relays with %u of %u gradients", (unsigned long long)i, ev.learner, leaf_fill[ev.learner], fanin);
+            if (ev.ts != ts) return fail(RUDRA_E_STATE, "event %llu: relay expects server timestamp %llu, server has %llu", (unsigned long long)i, (unsigned long long)ev.ts, (unsigned long long)ts);
+            if (queued % ps->c + fanin > ps->c) return fail(RUDRA_E_STATE, "event %llu: the relayed average does not fit the open group", (unsigned long long)i);
+            leaf_fill[ev.learner] = 0;
+            if ((queued += fanin) > RUDRA_QUEUE_CAP) return fail(RUDRA_E_QUEUE_FULL, "event %llu: queue full", (unsigned long long)i);
             break;
           case RUDRA_EV_STEP:
             if (queued < ps->c) return fail(RUDRA_E_STATE, "event %llu: update with %llu of %u gradients queued", (unsigned long long)i, (unsigned long long)queued, ps->c);
@@ -668,9 +876,30 @@ int64_t rudra_ps_run_events(rudra_ps* ps, const rudra_event* events, uint64_t co
     for (uint64_t i = 0; i < count; ++i) {
       const rudra_event& ev = events[i];
       switch (ev.kind) {
-        case RUDRA_EV_PUSH:
-          enqueue(ps, grads_dev[ev.learner], ev.pulled_ts, -1);
+        case RUDRA_EV_PUSH: {
+          Pending e{grads_dev[ev.learner], ev.pulled_ts, -1, 1u, false};
+          if (ps->push_mode == RUDRA_PUSH_COPY) {
+            if (int r = stage_device_copy(ps, e.grad, &e.slot)) return r;
+            e.grad = ps->slots[e.slot];
+          }
+          if (ps->fanin) {
+            ps->leaf_pending[ev.learner / ps->fanin].push_back(e);
+          } else {
+            ps->queue.push_back(e);
+            ps->counters[0] += 1;
+          }
           break;
+        }
+        case RUDRA_EV_RELAY: {
+          // The leaf shares this GPU with the root: it hands over its learners' raw vectors and the
+          // update kernel averages them on the way (no intermediate vector is written).
+          std::vector<Pending>& leaf = ps->leaf_pending[ev.learner];
+          uint64_t stamps[RUDRA_MAX_GROUP];
+          for (uint32_t l = 0; l < ps->fanin; ++l) stamps[l] = leaf[l].pulled_ts;
+          enqueue_group(ps, leaf.data(), ps->fanin, stamps, ps->fanin);
+          leaf.clear();
+          break;
+        }
         case RUDRA_EV_STEP:
           if (!window_has_room_for_update(ps, w, cap))
             if (int r = flush_window(ps, w)) return r;

@@ -44,6 +44,11 @@ struct rudra_sched {
   bool downcast;
   double spread;
 
+  uint32_t fanin;                       // learners per leaf of the server tree (Section 3.3); 0 = no tree
+  std::vector<uint32_t> at_leaf;        // gradients each leaf holds
+  std::vector<uint64_t> relayed;        // averages each leaf has sent up
+  uint64_t at_root = 0;                 // gradients that have reached the root (directly or averaged)
+
   uint64_t server_ts = 0;
   uint64_t handled = 0;                 // pushes handled so far
   std::vector<uint64_t> delivered_ts;   // timestamp of the weights in each learner's receive buffer
@@ -61,8 +66,9 @@ struct rudra_sched {
   std::vector<rudra_event> pending;     // events produced by the push being handled
   size_t pending_pos = 0;
 
-  rudra_sched(uint32_t lam, uint32_t n_, int mode_, uint64_t seed, double spread_, bool downcast_)
-      : lambda(lam), n(n_), c(lam / n_), mode(mode_), downcast(downcast_), spread(spread_),
+  rudra_sched(uint32_t lam, uint32_t n_, int mode_, uint64_t seed, double spread_, bool downcast_, uint32_t fanin_)
+      : lambda(lam), n(n_), c(lam / n_), mode(mode_), downcast(downcast_), spread(spread_), fanin(fanin_),
+        at_leaf(fanin_ ? lam / fanin_ : 0, 0), relayed(fanin_ ? lam / fanin_ : 0, 0),
         delivered_ts(lam, 0), in_use_ts(lam, 0), batches(lam, 0), order_rng(substream(seed, kPurposeOrder, 0)) {
     if (mode == RUDRA_SCHED_SOFTSYNC_TIMED) {
       time_rng.reserve(lam);
@@ -104,7 +110,21 @@ struct rudra_sched {
   // pullWeights is served.
   void on_push(uint32_t l, uint64_t tick) {
     add(RUDRA_EV_PUSH, l, in_use_ts[l], server_ts, batches[l]++, tick);
-    const bool closes_group = (++handled % c) == 0;
+    ++handled;
+    bool closes_group = false;
+    if (fanin == 0) {
+      closes_group = ++at_root % c == 0;
+    } else if (++at_leaf[l / fanin] == fanin) {   // the leaf is full: its average goes up now
+      const uint32_t leaf = l / fanin;
+      at_leaf[leaf] = 0;
+      add(RUDRA_EV_RELAY, leaf, 0, server_ts, relayed[leaf]++, tick);
+      at_root += fanin;
+      closes_group = at_root % c == 0;
+    }
+    finish_push(l, tick, closes_group);
+  }
+
+  void finish_push(uint32_t l, uint64_t tick, bool closes_group) {
     if (closes_group) add(RUDRA_EV_STEP, l, 0, ++server_ts, 0, tick);
 
     if (mode == RUDRA_SCHED_HARDSYNC) {
@@ -146,21 +166,42 @@ struct rudra_sched {
 
 extern "C" {
 
-rudra_sched* rudra_sched_create(uint32_t lambda, uint32_t n, int mode, uint64_t seed,
-                                double lognormal_sigma, int downcast) {
+rudra_sched* rudra_sched_create_tree(uint32_t lambda, uint32_t n, int mode, uint64_t seed,
+                                     double lognormal_sigma, int downcast, uint32_t fanin) {
   if (lambda == 0 || n == 0 || n > lambda) return nullptr;
   if (mode != RUDRA_SCHED_HARDSYNC && mode != RUDRA_SCHED_SOFTSYNC_ROUNDS && mode != RUDRA_SCHED_SOFTSYNC_TIMED)
     return nullptr;
   if (mode == RUDRA_SCHED_HARDSYNC && n != 1) return nullptr;
   if (!(lognormal_sigma >= 0.0) || !std::isfinite(lognormal_sigma)) return nullptr;
-  return new (std::nothrow) rudra_sched(lambda, n, mode, seed, lognormal_sigma, downcast != 0);
+  if (fanin != 0 && (lambda % fanin != 0 || (lambda / n) % fanin != 0)) return nullptr;
+  try {
+    return new rudra_sched(lambda, n, mode, seed, lognormal_sigma, downcast != 0, fanin);
+  } catch (...) {
+    return nullptr;
+  }
+}
+
+rudra_sched* rudra_sched_create(uint32_t lambda, uint32_t n, int mode, uint64_t seed,
+                                double lognormal_sigma, int downcast) {
+  return rudra_sched_create_tree(lambda, n, mode, seed, lognormal_sigma, downcast, 0);
+}
+
+int rudra_sched_on_pull(rudra_sched* s, uint32_t learner, uint64_t ts) {
+  if (!s || learner >= s->lambda) return RUDRA_E_INVAL;
+  if (ts > s->server_ts) return RUDRA_E_BAD_TS;
+  s->delivered_ts[learner] = s->in_use_ts[learner] = ts;
+  return 0;
 }
 
 void rudra_sched_destroy(rudra_sched* s) { delete s; }
 
 int64_t rudra_sched_next(rudra_sched* s, rudra_event* out, uint64_t count) {
   if (!s || (!out && count)) return RUDRA_E_INVAL;
-  for (uint64_t i = 0; i < count; ++i) out[i] = s->next();
+  try {
+    for (uint64_t i = 0; i < count; ++i) out[i] = s->next();
+  } catch (...) {
+    return RUDRA_E_NOMEM;
+  }
   return (int64_t)count;
 }
 

@@ -20,72 +20,13 @@
 // faster on B200 than a persistent grid-stride loop).  Successive launches sweep in alternating
 // directions: a launch starts on the tail the previous one just wrote, which is still in the
 // 126 MB L2, so those lines are neither re-read from HBM nor written back twice.
-#include <cuda_bf16.h>
-
 #include "kernels.cuh"
+#include "vec.cuh"
 
 namespace rudra {
 namespace {
 
-constexpr int kUnit = 8;   // weights per thread per unit
 constexpr uint64_t kSmallModel = 262144;   // below this many weights the one-weight-per-thread kernel runs
-
-struct alignas(32) F8 { float v[kUnit]; };
-
-__device__ __forceinline__ F8 ld8(const float* p) {
-  F8 r;
-  asm volatile("ld.global.L2::evict_last.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
-               : "l"(p));
-  return r;
-}
-
-__device__ __forceinline__ void st8(float* p, const F8& r) {
-  asm volatile("st.global.L2::evict_last.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
-               :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
-               : "memory");
-}
-
-// Pull destinations: plain write-back stores (measured 1 % faster on B200 than evict-first or
-// evict-last hints when half the traffic of a window is pull writes).
-__device__ __forceinline__ void st8_stream(float* p, const F8& r) {
-  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
-               :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
-               : "memory");
-}
-
-// One unit of one gradient stream, as loaded (fp32: 8 floats; bf16: 8 halves in 4 words).
-template <typename G> struct GradUnit;
-template <> struct GradUnit<float> {
-  F8 raw;
-  __device__ __forceinline__ void load(const void* base, uint64_t unit) {
-    const float* p = static_cast<const float*>(base) + unit * kUnit;
-    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=f"(raw.v[0]), "=f"(raw.v[1]), "=f"(raw.v[2]), "=f"(raw.v[3]), "=f"(raw.v[4]), "=f"(raw.v[5]), "=f"(raw.v[6]), "=f"(raw.v[7])
-                 : "l"(p));
-  }
-  __device__ __forceinline__ void zero() {
-#pragma unroll
-    for (int e = 0; e < kUnit; ++e) raw.v[e] = 0.f;
-  }
-  __device__ __forceinline__ float get(int e) const { return raw.v[e]; }
-  static __device__ __forceinline__ float scalar(const void* base, uint64_t k) { return static_cast<const float*>(base)[k]; }
-};
-template <> struct GradUnit<__nv_bfloat16> {
-  uint4 raw;
-  __device__ __forceinline__ void load(const void* base, uint64_t unit) {
-    raw = __ldcs(static_cast<const uint4*>(base) + unit);
-  }
-  __device__ __forceinline__ void zero() { raw = make_uint4(0u, 0u, 0u, 0u); }
-  // bf16 is the upper half of an fp32: widening is a shift, exact.
-  __device__ __forceinline__ float get(int e) const {
-    const uint32_t w = e < 2 ? raw.x : e < 4 ? raw.y : e < 6 ? raw.z : raw.w;
-    return __uint_as_float((e & 1) ? (w & 0xFFFF0000u) : (w << 16));
-  }
-  static __device__ __forceinline__ float scalar(const void* base, uint64_t k) {
-    return __uint_as_float((uint32_t)static_cast<const uint16_t*>(base)[k] << 16);
-  }
-};
 
 // The per-weight rule.  Momentum SGD: u = acc + (sum s) wd theta; v' = m v + u; theta' = theta - v'.
 // AdaGrad: g = acc + wd theta (acc already the weighted mean gradient); h' = h + g^2;
@@ -137,9 +78,9 @@ __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t uni
       if (!GUARD || u < nunits) st8_stream(p.dst[d] + u * kUnit, th[j]);
     }
   }
-  const uint32_t total = p.nupd * p.c;
-  uint32_t w = 0;            // update being accumulated
-  uint32_t left = p.c;       // gradients it still waits for
+  const uint32_t total = p.grad_end[p.nupd];
+  uint32_t w = 0;                    // update being accumulated
+  uint32_t last = p.grad_end[1];     // one past its last gradient vector
   for (uint32_t l0 = 0; l0 < total; l0 += DEPTH) {
     GradUnit<G> g[DEPTH][U];
 #pragma unroll
@@ -161,7 +102,7 @@ __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t uni
         for (int j = 0; j < U; ++j)
 #pragma unroll
           for (int e = 0; e < kUnit; ++e) acc[j][e] = fmaf(s, g[i][j].get(e), acc[j][e]);
-        if (--left == 0) {     // last gradient of update w: applyUpdate, then the pulls that follow it
+        if (l0 + i + 1 == last) {   // last gradient of update w: applyUpdate, then the pulls that follow it
           const float awd = p.awd[w], abar = p.abar[w];
 #pragma unroll
           for (int j = 0; j < U; ++j)
@@ -173,7 +114,7 @@ __device__ __forceinline__ void process_tile(const UpdateParams& p, uint64_t uni
               acc[j][e] = 0.f;
             }
           ++w;
-          left = p.c;
+          last = p.grad_end[w + 1];   // (the entry after the last update is never compared: the loop ends first)
           for (const uint32_t d1 = p.dst_end[w]; d < d1; ++d) {
 #pragma unroll
             for (int j = 0; j < U; ++j) {
@@ -214,7 +155,7 @@ __global__ void __launch_bounds__(THREADS) update_kernel(const __grid_constant__
     for (const uint32_t d1 = p.dst_end[0]; d < d1; ++d) p.dst[d][k] = th;
     for (uint32_t w = 0; w < p.nupd; ++w) {
       float acc = 0.f;
-      for (const uint32_t l1 = l + p.c; l < l1; ++l) acc = fmaf(p.scale[l], GradUnit<G>::scalar(p.grad[l], k), acc);
+      for (const uint32_t l1 = p.grad_end[w + 1]; l < l1; ++l) acc = fmaf(p.scale[l], GradUnit<G>::scalar(p.grad[l], k), acc);
       apply<OPT, STATE>(p, p.awd[w], p.abar[w], acc, th, s);
       for (const uint32_t d1 = p.dst_end[w + 1]; d < d1; ++d) p.dst[d][k] = th;
     }
@@ -236,8 +177,8 @@ __global__ void __launch_bounds__(THREADS) update_kernel_small(const __grid_cons
   float st = STATE ? p.state[k] : 0.f;
   uint32_t d = 0;
   for (const uint32_t d1 = p.dst_end[0]; d < d1; ++d) p.dst[d][k] = th;
-  const uint32_t total = p.nupd * p.c;
-  uint32_t w = 0, left = p.c;
+  const uint32_t total = p.grad_end[p.nupd];
+  uint32_t w = 0, last = p.grad_end[1];
   float acc = 0.f;
   for (uint32_t l0 = 0; l0 < total; l0 += DEPTH) {
     float g[DEPTH];
@@ -248,11 +189,11 @@ __global__ void __launch_bounds__(THREADS) update_kernel_small(const __grid_cons
     for (int i = 0; i < DEPTH; ++i) {
       if (l0 + i < total) {
         acc = fmaf(p.scale[l0 + i], g[i], acc);
-        if (--left == 0) {
+        if (l0 + i + 1 == last) {
           apply<OPT, STATE>(p, p.awd[w], p.abar[w], acc, th, st);
           acc = 0.f;
           ++w;
-          left = p.c;
+          last = p.grad_end[w + 1];
           for (const uint32_t d1 = p.dst_end[w]; d < d1; ++d) p.dst[d][k] = th;
         }
       }

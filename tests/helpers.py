@@ -20,6 +20,28 @@ def rel_err(got, want):
     return float(np.max(np.abs(got - want) / den)) if want.size else 0.0
 
 
+def adagrad_slack(h_oracle, abar, terms, gmax, eps=1e-8):
+    """Absolute error one AdaGrad step may add to a weight beyond the relative bar, per weight.
+
+    The step is abar * g / (sqrt(h) + eps) with h the running sum of squares including g^2; its
+    derivative with respect to g is at most abar / (sqrt(h) + eps).  An fp32 evaluation of g (a mean
+    of `terms` values of magnitude up to gmax plus the penalty) is off by up to about
+    (terms + 2) 2^-24 gmax, which the division amplifies where sqrt(h) is small -- in the first
+    steps, for the few weights whose gradient happens to be within a few hundred eps of zero.
+    h_oracle is the oracle's state after the step."""
+    delta = (terms + 2) * 2.0 ** -24 * gmax
+    return abar * delta / (np.sqrt(np.asarray(h_oracle, dtype=np.float64)) + eps)
+
+
+def rel_err_beyond(got, want, slack):
+    """rel_err after an absolute allowance ``slack`` (per weight) has been taken off the difference."""
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    rms = float(np.sqrt(np.mean(want * want)))
+    den = np.maximum(np.abs(want), max(rms, 1e-30))
+    return float(np.max(np.maximum(np.abs(got - want) - slack, 0.0) / den))
+
+
 def to_device(arr):
     """numpy -> CUDA tensor holding the same bytes (uint16 bf16 patterns travel as int16)."""
     import torch

@@ -8,7 +8,8 @@ import pytest
 from oracle import rudra_oracle as ora
 from paper_1509_04210_b200 import synth
 
-from helpers import REL_100_STEPS, REL_ONE_STEP, Pair, rel_err, run_workload, to_device, to_host
+from helpers import (REL_100_STEPS, REL_ONE_STEP, Pair, adagrad_slack, rel_err, rel_err_beyond, run_workload, to_device,
+                     to_host)
 
 pytestmark = pytest.mark.gpu
 
@@ -83,11 +84,19 @@ def test_policies_and_optimizer_terms(policy, momentum, wd):
 def test_adagrad_parity():
     N, lam, n = 33333, 8, 2
     pair = Pair(N, lam, n, 0.01, 0.0, 5e-4, optimizer=ora.OPT_ADAGRAD)
+    slack = np.zeros(N)
     for step in range(12):
         for l in range(4):
             pair.push(synth.gradient(N, l, step, 1e-2), pair.gpu.timestamp())
         assert pair.step() == 1
-        pair.compare(REL_ONE_STEP if step == 0 else REL_100_STEPS)
+        # the division by sqrt(h) + eps amplifies the fp32 rounding of the mean gradient where h is tiny
+        slack += adagrad_slack(pair.cpu.state(), pair.cpu.last_clock()["abar"], 4, 0.06)
+        th, st = pair.weights()
+        tol = REL_ONE_STEP if step == 0 else REL_100_STEPS
+        assert rel_err_beyond(th, pair.cpu.pull()[0], slack) <= tol
+        assert rel_err(st, pair.cpu.state()) <= tol
+    # the allowance is a sliver of the distance a weight travels (12 steps of about abar each) for all but a few
+    assert np.quantile(slack, 0.99) < 1e-3 * 12 * pair.cpu.last_clock()["abar"]
     pair.close()
 
 

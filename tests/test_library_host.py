@@ -53,7 +53,10 @@ def test_header_constants_match_binding():
                                                              rb.E_NOMEM)
     assert defs["RUDRA_HIST_BINS"] == rb.HIST_BINS
     assert (defs["RUDRA_EV_PUSH"], defs["RUDRA_EV_STEP"], defs["RUDRA_EV_PULL"], defs["RUDRA_EV_PULL_SKIP"],
-            defs["RUDRA_EV_BROADCAST"]) == (1, 2, 3, 4, 5)
+            defs["RUDRA_EV_BROADCAST"], defs["RUDRA_EV_RELAY"]) == (1, 2, 3, 4, 5, 6) == (
+        ora.PUSH, ora.STEP, ora.PULL, ora.PULL_SKIP, ora.BROADCAST, ora.RELAY)
+    assert (defs["RUDRA_OPT_PUSH_MODE"], defs["RUDRA_OPT_TREE_FANIN"], defs["RUDRA_PUSH_COPY"]) == (
+        rb.OPT_PUSH_MODE, rb.OPT_TREE_FANIN, rb.PUSH_COPY)
     assert defs["RUDRA_GRAD_BF16"] == rb.GRAD_BF16 == synth.GRAD_BF16
     assert (defs["RUDRA_SCHED_HARDSYNC"], defs["RUDRA_SCHED_SOFTSYNC_ROUNDS"], defs["RUDRA_SCHED_SOFTSYNC_TIMED"]) == (
         synth.HARDSYNC, synth.SOFTSYNC_ROUNDS, synth.SOFTSYNC_TIMED)
@@ -83,6 +86,63 @@ def test_scheduler_trace_equals_oracle_bit_for_bit(lam, n, mode, spread, downcas
     b = ora.OracleScheduler(lam, n, mode, seed, spread, downcast).run(count)
     assert a.tobytes() == b.tobytes()
     assert (a["kind"] == rb.EV_PUSH).sum() > count // 4
+
+
+TREE_CASES = [
+    (12, 2, rb.SCHED_SOFTSYNC_ROUNDS, 0.3, False, 3),
+    (54, 18, rb.SCHED_SOFTSYNC_ROUNDS, 0.3, False, 3),
+    (54, 3, rb.SCHED_SOFTSYNC_ROUNDS, 0.3, False, 6),
+    (128, 4, rb.SCHED_SOFTSYNC_ROUNDS, 0.3, True, 8),
+    (8, 1, rb.SCHED_HARDSYNC, 0.3, False, 4),
+    (60, 4, rb.SCHED_SOFTSYNC_TIMED, 0.3, False, 5),
+    (6, 2, rb.SCHED_SOFTSYNC_TIMED, 0.7, True, 1),
+]
+
+
+@pytest.mark.parametrize("lam,n,mode,spread,downcast,fanin", TREE_CASES)
+@pytest.mark.parametrize("seed", [synth.MASTER_SEED, 2**63 + 12345])
+def test_tree_scheduler_trace_equals_oracle_bit_for_bit(lam, n, mode, spread, downcast, fanin, seed):
+    # learners -> leaves -> root (Section 3.3): PUSH, RELAY, STEP and pull events in the same order
+    count = 20000
+    a = rb.Scheduler(lam, n, mode, seed, spread, downcast, fanin).next(count)
+    b = ora.OracleScheduler(lam, n, mode, seed, spread, downcast, fanin).run(count)
+    assert a.tobytes() == b.tobytes()
+    assert (a["kind"] == rb.EV_RELAY).sum() * fanin <= (a["kind"] == rb.EV_PUSH).sum()
+    assert (a["kind"] == rb.EV_RELAY).sum() > count // (8 * fanin)
+    with pytest.raises(ValueError):
+        rb.Scheduler(lam, n, mode, seed, spread, downcast, lam + 1)
+
+
+@pytest.mark.parametrize("mode,fanin", [(rb.SCHED_SOFTSYNC_ROUNDS, 0), (rb.SCHED_SOFTSYNC_TIMED, 0), (rb.SCHED_SOFTSYNC_ROUNDS, 2)])
+def test_reported_pulls_change_the_trace_the_same_way_on_both_sides(mode, fanin):
+    # learner 3 loses every second pull and reports the weights it really holds: its gradients are
+    # staler than the scheduler assumed.  Both schedulers must take the report the same way.
+    lam, n = 12, 3
+    a = rb.Scheduler(lam, n, mode, 77, 0.3, False, fanin)
+    b = ora.OracleScheduler(lam, n, mode, 77, 0.3, False, fanin)
+    held, lost, reported = 0, 0, 0
+    stale_seen = 0
+    for _ in range(6000):
+        ea, eb = a.next(1)[0], b.run(1)[0]
+        assert ea.tobytes() == eb.tobytes()
+        if int(ea["learner"]) != 3:
+            continue
+        if ea["kind"] == rb.EV_PUSH:
+            assert int(ea["pulled_ts"]) == held              # the push carries what the learner reported
+            stale_seen = max(stale_seen, int(ea["ts"]) - held)
+        elif ea["kind"] in (rb.EV_PULL, rb.EV_PULL_SKIP):
+            lost += 1
+            if lost % 2 == 0:
+                held = int(ea["ts"])
+            else:
+                assert a.on_pull(3, held) == 0 and b.on_pull(3, held) == 0
+                reported += 1
+    assert reported > 50 and stale_seen > n
+    with pytest.raises(rb.RudraError) as e:
+        a.on_pull(3, 10**9)                                  # weights that do not exist yet
+    assert e.value.code == rb.E_BAD_TS and b.on_pull(3, 10**9) == -2
+    with pytest.raises(rb.RudraError):
+        a.on_pull(lam, 0)
 
 
 def test_scheduler_is_incremental():
