@@ -281,7 +281,11 @@ def run_reference(args, w):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(w),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "cpu_model": cpu_model()},
+        "timed_seconds": dt, "timed_windows": done, "sample_fraction": frac,
+        "ms_per_step_note": "ms_per_step is 1000 / value, the time a full-size window would take at the sampled rate; "
+                            "the run itself timed %d windows of the sample in %.1f s" % (done, dt),
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -303,6 +307,174 @@ def workload_config(w):
 # ---------------------------------------------------------------------------------------------
 # the CUDA arm
 # ---------------------------------------------------------------------------------------------
+def cpu_model():
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    import platform
+
+    return platform.processor() or platform.machine()
+
+
+def batch_shape(w, batch):
+    """(updates, gradient vectors, weight copies) one backlog asks of the server."""
+    kinds = batch["kind"]
+    updates = int((kinds == EV_STEP).sum())
+    copies = int((kinds == EV_PULL).sum()) + w.lam * int((kinds == EV_BROADCAST).sum())
+    return updates, updates * w.c, copies
+
+
+class DeviceRun:
+    """One parameter server with everything resident in HBM, driven over a workload's event stream."""
+
+    def __init__(self, rb, torch, w, args, seed, stream, views=False):
+        self.rb, self.torch, self.w, self.stream, self.views = rb, torch, w, stream, views
+        N = w.nparams
+        self.nbufs = min(w.lam, args.buffers) if args.buffers else w.lam
+        self.bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype, seed) for l in range(self.nbufs)]
+        self.nslots = 0 if views else self.nbufs
+        self.slots = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(self.nslots)]
+        ps = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
+        ps.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
+        if ADAGRAD:
+            ps.set_option(rb.OPT_OPTIMIZER, rb.OPTIM_ADAGRAD)
+        ps.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
+        if views:
+            ps.enable_views(w.lam + 1)
+        ps.sync()
+        ps.set_stream(stream)
+        self.ps = ps
+        self.gtable = rb.pointer_table([self.bufs[l % self.nbufs] for l in range(w.lam)])
+        self.stable = None if views else rb.pointer_table([self.slots[l % self.nslots] for l in range(w.lam)])
+        self.pool = []
+
+    def events(self, count):
+        """Timing event pairs made (and recorded once) ahead of the timed region, so that none is created in it."""
+        for _ in range(count):
+            pair = (self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True))
+            pair[0].record(self.stream)
+            pair[1].record(self.stream)
+            self.pool.append(pair)
+
+    def pair(self):
+        if self.pool:
+            return self.pool.pop()
+        return self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True)
+
+    def messages(self, win, upd_events, pull_events=None):
+        """One message at a time through push / step / pull."""
+        ps, bufs, slots, stream = self.ps, self.bufs, self.slots, self.stream
+        for kind, learner, pulled_ts in zip(win["kind"].tolist(), win["learner"].tolist(), win["pulled_ts"].tolist()):
+            if kind == EV_PUSH:
+                ps.push(bufs[learner % self.nbufs], pulled_ts)
+            elif kind == EV_STEP:
+                e0, e1 = self.pair()
+                e0.record(stream)
+                ps.step()
+                e1.record(stream)
+                upd_events.append((e0, e1))
+            elif kind == EV_PULL:
+                if pull_events is None:
+                    ps.pull(slots[learner % self.nslots])
+                else:
+                    e0, e1 = self.pair()
+                    e0.record(stream)
+                    ps.pull(slots[learner % self.nslots])
+                    e1.record(stream)
+                    pull_events.append((e0, e1, 1))
+            elif kind == EV_BROADCAST:
+                if pull_events is None:
+                    ps.pull_many(slots)
+                else:
+                    e0, e1 = self.pair()
+                    e0.record(stream)
+                    ps.pull_many(slots)
+                    e1.record(stream)
+                    pull_events.append((e0, e1, len(slots)))
+
+    def backlog(self, chunk, W, timed, host_s):
+        """A backlog of update windows through one rudra_ps_run_events call."""
+        e0, e1 = self.pair()
+        e0.record(self.stream)
+        t0 = time.perf_counter()
+        self.ps.run_events(chunk, self.gtable, self.stable, W)
+        host_s.append(time.perf_counter() - t0)
+        e1.record(self.stream)
+        timed.append((e0, e1))
+
+    def close(self):
+        self.ps.close()
+        self.bufs, self.slots = [], []
+
+
+def timed_region(run, w, windows, warmup, steps, W, barrier, sampler_factory=None):
+    """Warm-up, then exactly ``steps`` update windows between two events.  With a backlog size W the
+    warm-up is rounded up to whole backlogs so that the timed backlogs start where a round of the
+    learners starts; the timed windows are handed over as backlogs of W (the last may be shorter)."""
+    torch, stream, ps = run.torch, run.stream, run.ps
+    warm = warmup if W == 0 else -(-warmup // W) * W
+    wins = windows[: warm + steps]
+    assert len(wins) == warm + steps
+    if W == 0:
+        warm_batches, batches = wins[:warm], wins[warm:]
+    else:
+        warm_batches = [np.concatenate(wins[i:i + W]) for i in range(0, warm, W)]
+        batches = [np.concatenate(wins[i:i + W]) for i in range(warm, warm + steps, W)]
+    shapes = [batch_shape(w, b) for b in batches]
+    junk, host_s = [], []
+    for b in warm_batches:
+        run.messages(b, junk) if W == 0 else run.backlog(b, W, junk, [])
+    run.pool.extend(junk)
+    run.events((steps if W == 0 else len(batches)) + 4)
+    barrier()
+    sampler = sampler_factory() if sampler_factory else None
+    if sampler:
+        sampler.start()
+    c0 = ps.counters()
+    start, end = run.pair()
+    timed = []
+    start.record(stream)
+    for b in batches:
+        run.messages(b, timed) if W == 0 else run.backlog(b, W, timed, host_s)
+    end.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    c1 = ps.counters()
+    return {
+        "ms": start.elapsed_time(end), "launch_ms": [a.elapsed_time(b) for a, b in timed], "shapes": shapes,
+        "host_us": [1e6 * t for t in host_s], "warmup_done": warm, "clocks": clocks,
+        "launches": c1["launches"] - c0["launches"], "pulls": c1["pulls"] - c0["pulls"],
+        "copies": c1["weight_copies"] - c0["weight_copies"], "batches": len(batches), "views": run.views,
+    }
+
+
+def launch_shapes(w, N, W, region):
+    """Per launch shape (number of updates a run_events call carried): launches, device time and the
+    algorithmic bytes of one call.  A call is one fused launch; where the library splits a broadcast
+    off into a copy launch (one more read of the weights) the extra launches are spread evenly."""
+    g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
+    sb = state_bytes(w)
+    extra_per_call = max(0, region["launches"] - region["batches"]) / max(region["batches"], 1)
+    out = {}
+    total_updates = max(1, sum(u for u, _, _ in region["shapes"]))
+    for (updates, vectors, copies), ms in zip(region["shapes"], region["launch_ms"]):
+        if region.get("views"):   # shared versions: a version is written once however many learners take it
+            copies = region["copies"] * updates / total_updates
+        rec = out.setdefault(updates, {"updates": updates, "gradient_vectors": vectors, "weight_copies": copies, "launches": 0,
+                                       "ms": 0.0})
+        rec["launches"] += 1
+        rec["ms"] += ms
+        rec["bytes_per_launch"] = float(N) * (vectors * g + sb + 4 * copies + 4 * extra_per_call)
+    for rec in out.values():
+        rec["avg_launch_us"] = 1e3 * rec.pop("ms") / rec["launches"]
+        rec["gbs"] = rec["bytes_per_launch"] / (rec["avg_launch_us"] * 1e-6) / 1e9
+    return out
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -328,114 +500,36 @@ def run_ours(args, w):
     N = w.nparams
     seed = replicas.replica_seed(synth.MASTER_SEED, rank)
     stream = torch.cuda.Stream()
-    nbufs = min(w.lam, args.buffers) if args.buffers else w.lam
-    bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype, seed) for l in range(nbufs)]
     views = args.pull == "views"
-    nslots = 0 if views else nbufs
-    slots = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(nslots)]
-    ps = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
-    ps.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
-    if args.optimizer == "adagrad":
-        ps.set_option(rb.OPT_OPTIMIZER, rb.OPTIM_ADAGRAD)
-    ps.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
-    if views:
-        ps.enable_views(w.lam + 1)
-    ps.sync()
-    ps.set_stream(stream)
-    extra_steps = 0 if (args.window == 0 or args.pull == "views") else min(args.steps, 216)
-    windows = make_windows(w, args.warmup + args.steps + extra_steps)
-    extra_windows = windows[args.warmup + args.steps:]
-    windows = windows[: args.warmup + args.steps]
     W = default_window(w, views) if args.window < 0 else args.window
     if views and W == 0:
         raise SystemExit("--pull views is served through rudra_ps_run_events: use --window >= 1")
-    gtable = rb.pointer_table([bufs[l % nbufs] for l in range(w.lam)])
-    stable = None if views else rb.pointer_table([slots[l % nslots] for l in range(w.lam)])
-
-    event_pool = []
-
-    def new_events():
-        """A pair of timing events; pairs made before the timed region are re-used inside it so that
-        no event is created between launches."""
-        if event_pool:
-            return event_pool.pop()
-        return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-
-    def fill_event_pool(count):
-        for _ in range(count):
-            pair = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-            pair[0].record(stream)      # the first record creates the underlying event
-            pair[1].record(stream)
-            event_pool.append(pair)
-
-    def run_messages(win, timed):
-        """One message at a time through push / step / pull (--window 0)."""
-        for kind, learner, pulled_ts in zip(win["kind"].tolist(), win["learner"].tolist(), win["pulled_ts"].tolist()):
-            if kind == EV_PUSH:
-                ps.push(bufs[learner % nbufs], pulled_ts)
-            elif kind == EV_STEP:
-                e0, e1 = new_events()
-                e0.record(stream)
-                ps.step()
-                e1.record(stream)
-                timed.append((e0, e1))
-            elif kind == EV_PULL:
-                ps.pull(slots[learner % nslots])
-            elif kind == EV_BROADCAST:
-                ps.pull_many(slots)
-
-    def run_backlog(chunk, timed):
-        """A backlog of W update windows through run_events: one launch when the tables allow."""
-        e0, e1 = new_events()
-        e0.record(stream)
-        ps.run_events(chunk, gtable, stable, W)
-        e1.record(stream)
-        timed.append((e0, e1))
-
-    def prepare(wins):
-        """The messages as the server receives them: single windows, or backlogs of W windows."""
-        if W == 0:
-            return wins
-        return [np.concatenate(wins[i:i + W]) for i in range(0, len(wins), W)]
-
-    def run_all(batches, timed):
-        for b in batches:
-            (run_messages if W == 0 else run_backlog)(b, timed)
-
-    warm_batches, timed_batches = prepare(windows[: args.warmup]), prepare(windows[args.warmup:])
-    run_all(warm_batches, [])
-    fill_event_pool(args.steps + 2 if W == 0 else len(timed_batches) + 2)
-    barrier()
-    sampler = ClockSampler(visible_gpu_index(local_rank))
-    sampler.start()
-    c0 = ps.counters()
-    start, end = new_events()
-    timed = []
-    start.record(stream)
-    run_all(timed_batches, timed)
-    end.record(stream)
-    barrier()
-    clocks = sampler.stop()
-    c1 = ps.counters()
-    ms = start.elapsed_time(end)
-    launch_ms = [a.elapsed_time(b) for a, b in timed]
+    run = DeviceRun(rb, torch, w, args, seed, stream, views)
+    ps, bufs, slots, nbufs = run.ps, run.bufs, run.slots, run.nbufs
+    warm_done = args.warmup if W == 0 else -(-args.warmup // W) * W
+    extra_steps = 0 if (W == 0 or views) else min(args.steps, 216)
+    windows = make_windows(w, warm_done + args.steps + extra_steps)
+    extra_windows = windows[warm_done + args.steps:]
+    region = timed_region(run, w, windows, args.warmup, args.steps, W, barrier,
+                          lambda: ClockSampler(visible_gpu_index(local_rank)))
+    ms, launch_ms, clocks = region["ms"], region["launch_ms"], region["clocks"]
     kern_ms = float(sum(launch_ms))
-    upd_ms = kern_ms / max(len(timed), 1)
-    launches = c1["launches"] - c0["launches"]
-    pulls = c1["pulls"] - c0["pulls"]
-    copies = c1["weight_copies"] - c0["weight_copies"]
+    launches, pulls, copies = region["launches"], region["pulls"], region["copies"]
+    g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
+    sb = state_bytes(w)
 
     # The same server, continuing the same event stream, driven one message at a time (push, step,
-    # pull as separate calls and launches): the unbatched figure beside the backlog figure.
-    single = None
-    if extra_steps and W != 0:
-        fill_event_pool(extra_steps + 2)
-        sev = []
+    # pull as separate calls and launches): the unbatched figure beside the backlog figure, and the
+    # launch times of the copy kernel that serves a pull by itself.
+    single, pull_roof = None, None
+    if extra_steps:
+        run.events(2 * extra_steps + len(extra_windows) * (w.c + 1) + 4)
+        sev, pev = [], []
         barrier()
-        s0, s1 = new_events()
+        s0, s1 = run.pair()
         s0.record(stream)
         for win in extra_windows:
-            run_messages(win, sev)
+            run.messages(win, sev, pev)
         s1.record(stream)
         barrier()
         sms = replicas.max_over_ranks([s0.elapsed_time(s1)], device="cuda")[0]
@@ -443,21 +537,29 @@ def run_ours(args, w):
         single = {"value": replicas.whole_job_rate(extra_steps, world, sms), "unit": UNIT, "steps": extra_steps,
                   "update_kernel_us": upd_us,
                   "update_kernel_gbs": update_bytes_per_param(w) * N / (upd_us * 1e-6) / 1e9}
+        if pev:
+            ndst = pev[0][2]
+            pull_us = 1e3 * float(np.mean([a.elapsed_time(b) for a, b, k in pev if k == ndst]))
+            pull_roof = {"us": pull_us, "ndst": ndst, "launches": sum(1 for x in pev if x[2] == ndst),
+                         "bytes": float(N) * (4 + 4 * ndst)}
 
-    # What HBM delivers on this GPU, in this run, for the same mix of reads and writes as one launch
-    # of the dominant kernel: a probe kernel that only streams that many vectors in and out.
+    shapes = launch_shapes(w, N, W, region) if W != 0 else {}
+    full = shapes.get(W) or (shapes[max(shapes)] if shapes else None)
+
+    # What HBM delivers on this GPU, in this run, for the same mix of reads and writes as one
+    # full-window launch of the dominant kernel: a probe kernel that only streams that many vectors
+    # in and out (the probe's tables hold 64 of each).
     mix = None
-    if W >= 1 and not views and w.grad_dtype == synth.GRAD_F32 and N * 8 > 126e6 and nbufs == w.lam:
-        per_launch = max(1, args.steps // max(len(timed), 1))
-        nr = min(64, per_launch * w.c + state_bytes(w) // 8)
-        nw = min(64, int(round(copies / max(len(timed), 1))) + state_bytes(w) // 8)
+    if full and not views and w.grad_dtype == synth.GRAD_F32 and N * 8 > 126e6 and nbufs == w.lam:
+        nr = min(64, full["gradient_vectors"] + sb // 8)
+        nw = min(64, full["weight_copies"] + sb // 8)
         extra = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(4)]
         srcs = (bufs + extra[:2])[-nr:] if nr <= len(bufs) + 2 else None
         dsts = (slots + extra[2:])[-nw:] if nw <= len(slots) + 2 else None
         if srcs and dsts:
             for _ in range(3):
                 probe.stream_probe(srcs, dsts, N, stream)
-            p0, p1 = new_events()
+            p0, p1 = run.pair()
             reps = 10
             p0.record(stream)
             for _ in range(reps):
@@ -465,9 +567,11 @@ def run_ours(args, w):
             p1.record(stream)
             torch.cuda.synchronize()
             mix = {"gbs": 4.0 * N * (nr + nw) * reps / (p0.elapsed_time(p1) * 1e-3) / 1e9, "reads": nr, "writes": nw,
+                   "launch_reads": full["gradient_vectors"] + sb // 8, "launch_writes": full["weight_copies"] + sb // 8,
                    "launches": reps,
-                   "how": "rudra_stream_probe: the same number of vectors streamed in and out, same access shape, no arithmetic"}
-        del extra
+                   "how": "rudra_stream_probe (librudra_probe.so): that many vectors streamed in and out, same access "
+                          "shape, no arithmetic; its tables hold 64 of each"}
+        del extra, srcs, dsts
 
     e2e_ms, e2e_steps, h0, h1 = float('nan'), 0, None, None
     if not args.kernel_only:
@@ -519,43 +623,80 @@ def run_ours(args, w):
         h1 = ps2.counters()
         e2e_ms = s2.elapsed_time(e2)
         ps2.close()
+        del hg, hdst
 
-    ms, e2e_ms, upd_ms = replicas.max_over_ranks([ms, e2e_ms, upd_ms], device="cuda")
+    ms, e2e_ms = replicas.max_over_ranks([ms, e2e_ms], device="cuda")
+
+    # the paper's other model shape and the broadcast-heavy shape, short runs on the same GPU
+    others = None
+    if world == 1 and w.name == "imagenet" and not args.kernel_only and not args.no_other_workloads:
+        run.close()
+        del bufs, slots
+        torch.cuda.empty_cache()
+        others = {}
+        for name, osteps, owarm in (("cifar10", 6000, 300), ("stress", 40, 4)):
+            ow = synth.WORKLOADS[name]
+            orun = DeviceRun(rb, torch, ow, args, seed, stream)
+            oW = default_window(ow)
+            owin = make_windows(ow, -(-owarm // oW) * oW + osteps)
+            reg = timed_region(orun, ow, owin, owarm, osteps, oW, barrier)
+            og = 2 if ow.grad_dtype == synth.GRAD_BF16 else 4
+            osb = 16 if ow.momentum else 8
+            obytes = sum(b["bytes_per_launch"] * b["launches"] for b in launch_shapes(ow, ow.nparams, oW, reg).values())
+            others[name] = {
+                "value": osteps / (reg["ms"] * 1e-3), "unit": UNIT, "steps": osteps, "warmup": reg["warmup_done"],
+                "nparams": ow.nparams, "lambda": ow.lam, "n": ow.n, "c": ow.c,
+                "grad_dtype": "bf16" if ow.grad_dtype == synth.GRAD_BF16 else "f32", "window": oW,
+                "bytes_per_param_per_step": obytes / ow.nparams / osteps,
+                "hbm_gbs": obytes / (reg["ms"] * 1e-3) / 1e9,
+                "gpu_launches": reg["launches"], "avg_launch_us": 1e3 * float(np.mean(reg["launch_ms"])),
+                "host_us_per_call": float(np.median(reg["host_us"])),
+                "roofline_claim": ow.nparams * 8 > 126e6,
+            }
+            del og, osb
+            orun.close()
+            del orun
+            torch.cuda.empty_cache()
 
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
-        g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
         # bytes the whole path must move per step: every gradient once, weights/state per launch, pulls
-        sb = state_bytes(w)
         if W == 0:
             path_bytes = N * (args.steps * (w.c * g + sb) + 8 * pulls)
+            kern_bytes = float(N * args.steps * (w.c * g + sb))     # the timed launches are the update kernels only
+            achieved = kern_bytes / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else float("nan")
+            roof_launches, roof_us, roof_bytes = len(launch_ms), 1e3 * kern_ms / max(len(launch_ms), 1), kern_bytes / max(len(launch_ms), 1)
+            label = "update_kernel (fused sumGradients + applyUpdate), one update per launch"
         else:
-            # every call makes one launch that carries its updates (weights and state read and
-            # written once); launches beyond that are copy kernels the library split off for a
-            # broadcast (one more read of the weights each)
-            update_launches = min(launches, len(timed))
-            path_bytes = N * (args.steps * w.c * g + update_launches * sb + 4 * (launches - update_launches) + 4 * copies)
-        # the timed launches: with a backlog every launch of the region (so their bytes are the whole
-        # path's), one message at a time only the update kernels
-        kern_bytes = float(path_bytes if W != 0 else N * args.steps * (w.c * g + sb))
-        achieved = kern_bytes / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else float("nan")
+            path_bytes = sum(b["bytes_per_launch"] * b["launches"] for b in shapes.values())
+            achieved, roof_launches, roof_us, roof_bytes = full["gbs"], full["launches"], full["avg_launch_us"], full["bytes_per_launch"]
+            label = "update_kernel (fused sumGradients + applyUpdate), %d-update window with its %d pulls%s" % (
+                full["updates"], full["weight_copies"],
+                "" if launches == region["batches"] else " + the copy kernel the library splits off for a broadcast")
         value = replicas.whole_job_rate(args.steps, world, ms)
         cfg = workload_config(w)
         cfg["parallelism"] = "replicas x%d (one independent server per GPU)" % world
         cfg["window"] = W
+        cfg["warmup_done"] = region["warmup_done"]
         cfg["pull"] = ("zero-copy: learners share a pointer to the version they pulled (rudra_ps_enable_views)" if views
                        else "copy into each learner's slot")
         cfg["window_note"] = ("messages handled one at a time (push / step / pull)" if W == 0 else
-                              "backlog of %d update windows per rudra_ps_run_events call" % W)
+                              "backlog of %d update windows per rudra_ps_run_events call; warm-up rounded up to whole backlogs" % W)
+        other_shapes = [b for k, b in sorted(shapes.items()) if b is not full]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None,
+            "dtype": "f32" if w.grad_dtype == synth.GRAD_F32 else "f32 arithmetic on bf16 gradients (widened exactly)",
+            "data": "synthetic",
             "config": cfg,
             "hbm_gbs_whole_path": path_bytes / (ms * 1e-3) / 1e9,
             "bytes_per_param_per_step": path_bytes / N / args.steps,
             "pulls_per_step": pulls / args.steps,
             "weight_copies_per_step": copies / args.steps,
+            "host_us_per_call": None if not region["host_us"] else {
+                "call": "rudra_ps_run_events through the Python binding", "median": float(np.median(region["host_us"])),
+                "max": float(max(region["host_us"])), "calls": len(region["host_us"])},
             "one_message_at_a_time": single,
             "gpu_launches": launches,
             "clocks": clocks,
@@ -565,36 +706,45 @@ def run_ours(args, w):
                 "d2h_bytes_per_step": (h1["d2h_bytes"] - h0["d2h_bytes"]) // e2e_steps,
             },
             "roofline": {
-                "kernel": "update_kernel (fused sumGradients + applyUpdate%s)%s" % (
-                    "" if W == 0 else ", %d-update window with its pulls" % W,
-                    "" if W == 0 or launches == len(timed) else " + the copy kernel the library splits off for a broadcast"),
+                "kernel": label,
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_kind": "of %s" % peak_kind, "launches_timed": len(timed), "avg_launch_us": upd_ms * 1e3,
-                "bytes_per_launch": kern_bytes / max(len(timed), 1),
+                "peak_kind": "of %s" % peak_kind, "launches_timed": roof_launches, "avg_launch_us": roof_us,
+                "bytes_per_launch": roof_bytes,
                 "launch_us": None if not launch_ms else {
-                    "min": 1e3 * min(launch_ms), "median": 1e3 * float(np.median(launch_ms)), "max": 1e3 * max(launch_ms),
-                    "first_tenth": 1e3 * float(np.mean(launch_ms[: max(1, len(launch_ms) // 10)])),
-                    "last_tenth": 1e3 * float(np.mean(launch_ms[-max(1, len(launch_ms) // 10):]))},
+                    "min": 1e3 * min(launch_ms), "median": 1e3 * float(np.median(launch_ms)), "max": 1e3 * max(launch_ms)},
                 "frac_of_8TBs_datasheet": achieved / 8000.0,
-                "traffic": ncu_traffic(w.name, W, N),
+                "traffic": None if (W == 0 or not full) else ncu_traffic(w.name, full["updates"], N),
                 "mix_ceiling": mix,
                 "frac_of_mix_ceiling": None if not mix else achieved / mix["gbs"],
+                "other_launch_shapes": other_shapes,
             },
+            "roofline_pull": None if not pull_roof else {
+                "kernel": "snapshot_kernel (pullWeights: one read of the weights, %d written cop%s)" % (
+                    pull_roof["ndst"], "y" if pull_roof["ndst"] == 1 else "ies"),
+                "bound": "hbm", "achieved": pull_roof["bytes"] / (pull_roof["us"] * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
+                "frac": pull_roof["bytes"] / (pull_roof["us"] * 1e-6) / 1e9 / peak, "peak_kind": "of %s" % peak_kind,
+                "launches_timed": pull_roof["launches"], "avg_launch_us": pull_roof["us"],
+                "bytes_per_launch": pull_roof["bytes"], "traffic": None,
+                "where": "the one-message-at-a-time leg of this run: every pull a launch of its own",
+            },
+            "other_workloads": others,
         }
         if world == 1 and not args.no_cpu_baseline and not args.kernel_only:
             from oracle import rudra_oracle as ora
 
             ora.build()
             nh = min(w.lam, 6)
+            hostg = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype, seed) for l in range(nh)]
             grads = [t.cpu().numpy() if w.grad_dtype == synth.GRAD_F32 else t.view(torch.int16).cpu().numpy().view(np.uint16)
-                     for t in bufs[:nh]]
+                     for t in hostg]
+            del hostg
             done, dt = oracle_run(w, windows, N, grads, warmup=1, budget_s=12.0, max_windows=args.steps,
                                   adagrad=args.optimizer == "adagrad")
             line["cpu_baseline"] = {
                 "value": done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
                 "sample": "%d full-size update windows of the same event stream (%d distinct gradient buffers), %.1f s"
                           % (done, nh, dt),
-                "host_cores_available": os.cpu_count(),
+                "host_cores_available": os.cpu_count(), "cpu_model": cpu_model(),
             }
             cores = os.cpu_count() or 1
             if cores > 1:
@@ -606,7 +756,8 @@ def run_ours(args, w):
                               % (done_all, dt_all),
                 }
         print(json.dumps(line), flush=True)
-    ps.close()
+    if others is None:
+        run.close()
     if world > 1:
         dist.destroy_process_group()
 
@@ -657,6 +808,8 @@ def main():
     ap.add_argument("--probe-mixes", action="store_true",
                     help="print what HBM delivers for several mixes of reads and writes (no bench line) and exit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the short cifar10 and stress runs that the default workload's line carries")
     ap.add_argument("--kernel-only", action="store_true",
                     help="device-resident timed region only: no end-to-end leg, no CPU baseline (profiler captures)")
     ap.add_argument("--nparams", type=int, default=0,
