@@ -47,7 +47,7 @@ def kernel_sources_sha():
     import hashlib
 
     h = hashlib.sha256()
-    for f in ("update.cu", "kernels.cuh"):
+    for f in ("update.cu", "kernels.cuh", "vec.cuh"):
         with open(os.path.join(ROOT, "paper_1509_04210_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -88,19 +88,19 @@ def update_bytes_per_param(w):
 EV_PUSH, EV_STEP, EV_PULL, EV_PULL_SKIP, EV_BROADCAST = 1, 2, 3, 4, 5
 
 
-def make_windows(w, count, seed=synth.MASTER_SEED, from_oracle=False):
+def make_windows(w, count, seed=synth.MASTER_SEED, from_oracle=False, fanin=0):
     """Event windows (arrays of event records): a window runs from the first push of a group to
     the last pull before the next group's first push.  The CUDA arm takes the events from the
     library's scheduler, the reference arm from the oracle's."""
     if from_oracle:
         from oracle import rudra_oracle as ora
 
-        osched = ora.OracleScheduler(w.lam, w.n, w.mode, seed, w.lognormal_sigma, w.downcast)
+        osched = ora.OracleScheduler(w.lam, w.n, w.mode, seed, w.lognormal_sigma, w.downcast, fanin)
         more = lambda k: osched.run(k)
     else:
         from paper_1509_04210_b200 import binding as rb
 
-        sched = rb.Scheduler(w.lam, w.n, w.mode, seed, w.lognormal_sigma, w.downcast)
+        sched = rb.Scheduler(w.lam, w.n, w.mode, seed, w.lognormal_sigma, w.downcast, fanin)
         more = lambda k: sched.next(k)
     windows, cur, stepped = [], [], False
     while len(windows) < count:
@@ -331,7 +331,7 @@ def batch_shape(w, batch):
 class DeviceRun:
     """One parameter server with everything resident in HBM, driven over a workload's event stream."""
 
-    def __init__(self, rb, torch, w, args, seed, stream, views=False):
+    def __init__(self, rb, torch, w, args, seed, stream, views=False, fanin=0):
         self.rb, self.torch, self.w, self.stream, self.views = rb, torch, w, stream, views
         N = w.nparams
         self.nbufs = min(w.lam, args.buffers) if args.buffers else w.lam
@@ -345,6 +345,8 @@ class DeviceRun:
         ps.set_weights(synth.device_initial_weights(N, w.theta_std, seed))
         if views:
             ps.enable_views(w.lam + 1)
+        if fanin:
+            ps.set_option(rb.OPT_TREE_FANIN, fanin)   # learners -> leaves -> this server (Section 3.3)
         ps.sync()
         ps.set_stream(stream)
         self.ps = ps
@@ -504,11 +506,13 @@ def run_ours(args, w):
     W = default_window(w, views) if args.window < 0 else args.window
     if views and W == 0:
         raise SystemExit("--pull views is served through rudra_ps_run_events: use --window >= 1")
-    run = DeviceRun(rb, torch, w, args, seed, stream, views)
+    if args.tree and W == 0:
+        raise SystemExit("--tree is served through rudra_ps_run_events: use --window >= 1")
+    run = DeviceRun(rb, torch, w, args, seed, stream, views, args.tree)
     ps, bufs, slots, nbufs = run.ps, run.bufs, run.slots, run.nbufs
     warm_done = args.warmup if W == 0 else -(-args.warmup // W) * W
-    extra_steps = 0 if (W == 0 or views) else min(args.steps, 216)
-    windows = make_windows(w, warm_done + args.steps + extra_steps)
+    extra_steps = 0 if (W == 0 or views or args.tree) else min(args.steps, 216)
+    windows = make_windows(w, warm_done + args.steps + extra_steps, fanin=args.tree)
     extra_windows = windows[warm_done + args.steps:]
     region = timed_region(run, w, windows, args.warmup, args.steps, W, barrier,
                           lambda: ClockSampler(visible_gpu_index(local_rank)))
@@ -629,7 +633,7 @@ def run_ours(args, w):
 
     # the paper's other model shape and the broadcast-heavy shape, short runs on the same GPU
     others = None
-    if world == 1 and w.name == "imagenet" and not args.kernel_only and not args.no_other_workloads:
+    if world == 1 and w.name == "imagenet" and not args.kernel_only and not args.no_other_workloads and not args.tree:
         run.close()
         del bufs, slots
         torch.cuda.empty_cache()
@@ -657,6 +661,40 @@ def run_ours(args, w):
             orun.close()
             del orun
             torch.cuda.empty_cache()
+        # the same ImageNet-scale stream behind the two-level server tree of Section 3.3 (18 leaves of 3
+        # learners on this GPU, their averaging fused into the root's launch), and the leaf's own kernel
+        k = 3
+        trun = DeviceRun(rb, torch, w, args, seed, stream, fanin=k)
+        tsteps, twarm = min(args.steps, 360), W
+        treg = timed_region(trun, w, make_windows(w, twarm + tsteps, fanin=k), twarm, tsteps, W, barrier)
+        tbytes = sum(b["bytes_per_launch"] * b["launches"] for b in launch_shapes(w, N, W, treg).values())
+        avg = torch.empty(N, dtype=torch.float32, device="cuda")
+        for i in range(3):
+            rb.leaf_average(trun.bufs[3 * i: 3 * i + k], w.grad_dtype, N, avg, stream)
+        l0, l1 = trun.pair()
+        reps = 18
+        l0.record(stream)
+        for i in range(reps):
+            rb.leaf_average(trun.bufs[3 * (i % 18): 3 * (i % 18) + k], w.grad_dtype, N, avg, stream)
+        l1.record(stream)
+        torch.cuda.synchronize()
+        leaf_us = 1e3 * l0.elapsed_time(l1) / reps
+        peak_now = measured_hbm_peak()[0]
+        others["imagenet_tree_fanin3"] = {
+            "value": tsteps / (treg["ms"] * 1e-3), "unit": UNIT, "steps": tsteps, "window": W, "fanin": k,
+            "relay": "leaves share the root's GPU: raw gradients handed over, averaged inside the update kernel",
+            "bytes_per_param_per_step": tbytes / N / tsteps, "hbm_gbs": tbytes / (treg["ms"] * 1e-3) / 1e9,
+            "gpu_launches": treg["launches"], "avg_launch_us": 1e3 * float(np.mean(treg["launch_ms"])),
+            "host_us_per_call": float(np.median(treg["host_us"])),
+            "roofline_leaf": {
+                "kernel": "leaf_average_kernel (a leaf's mean of its %d learners' gradients, one float vector out)" % k,
+                "bound": "hbm", "achieved": float(N) * (k * g + 4) / (leaf_us * 1e-6) / 1e9, "peak": peak_now, "unit": "GB/s",
+                "frac": float(N) * (k * g + 4) / (leaf_us * 1e-6) / 1e9 / peak_now, "launches_timed": reps,
+                "avg_launch_us": leaf_us, "bytes_per_launch": float(N) * (k * g + 4), "traffic": None},
+        }
+        trun.close()
+        del trun, avg
+        torch.cuda.empty_cache()
 
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
@@ -790,6 +828,36 @@ def run_probe_mixes(args, w):
               % (nr, nw, nw / (nr + nw), us, 4.0 * N * (nr + nw) / us * 1e-3), flush=True)
 
 
+def run_leaf_average(args, w):
+    """--leaf-average K: the leaf's averaging kernel alone on the workload's vector length (no bench line)."""
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    N, k = w.nparams, args.leaf_average
+    g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
+    nbuf = max(k, min(54, int(6e9 // (N * g))) // k * k)
+    bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype) for l in range(nbuf)]
+    avg = torch.empty(N, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    groups = [bufs[i:i + k] for i in range(0, nbuf, k)]
+    for grp in groups[:3]:
+        rb.leaf_average(grp, w.grad_dtype, N, avg, stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 3 * len(groups)
+    e0.record(stream)
+    for i in range(reps):
+        rb.leaf_average(groups[i % len(groups)], w.grad_dtype, N, avg, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us = 1e3 * e0.elapsed_time(e1) / reps
+    peak, kind = measured_hbm_peak()
+    print(json.dumps({"kernel": "leaf_average_kernel", "nparams": N, "k": k, "grad_bytes": g, "launches": reps,
+                      "avg_launch_us": us, "bytes_per_launch": float(N) * (k * g + 4),
+                      "gbs": float(N) * (k * g + 4) / (us * 1e-6) / 1e9, "peak": peak, "peak_kind": kind,
+                      "frac": float(N) * (k * g + 4) / (us * 1e-6) / 1e9 / peak}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -805,6 +873,10 @@ def main():
                     help="copy: every pull writes the learner's own slot; views: zero-copy shared weight versions")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adagrad"],
                     help="momentum SGD with weight decay (Section 4.2) or AdaGrad at the server (Section 5.5)")
+    ap.add_argument("--tree", type=int, default=0, metavar="FANIN",
+                    help="learners send to leaves of a two-level server tree (Section 3.3), FANIN learners per leaf")
+    ap.add_argument("--leaf-average", type=int, default=0, metavar="K",
+                    help="time the leaf's averaging kernel for K gradients per leaf (no bench line) and exit")
     ap.add_argument("--probe-mixes", action="store_true",
                     help="print what HBM delivers for several mixes of reads and writes (no bench line) and exit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -837,6 +909,9 @@ def main():
         w = dataclasses.replace(w, name=w.name + "@%d" % args.nparams, nparams=args.nparams)
     if args.probe_mixes:
         run_probe_mixes(args, w)
+        return
+    if args.leaf_average:
+        run_leaf_average(args, w)
         return
     if args.impl == "reference":
         run_reference(args, w)

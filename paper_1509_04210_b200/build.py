@@ -36,6 +36,7 @@ def _compile(path, sources, verbose):
     nvcc = os.environ.get("NVCC", "nvcc")
     tmp = path + ".tmp.%d" % os.getpid()
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-I", _INCLUDE, "-o", tmp]
+    cmd += os.environ.get("RUDRA_NVCC_DEFINES", "").split()   # e.g. "-DRUDRA_MID_THREADS=128" for a tile sweep
     cmd += [os.path.join(_CSRC, s) for s in sources]
     subprocess.check_call(cmd)
     os.replace(tmp, path)

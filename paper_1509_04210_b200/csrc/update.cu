@@ -28,6 +28,22 @@ namespace {
 
 constexpr uint64_t kSmallModel = 262144;   // below this many weights the one-weight-per-thread kernel runs
 
+// Tile shape for vectors between kSmallModel and ~4.8 M weights (build-time knobs; the defaults
+// are the fastest of a sweep over 32..256 threads and 4..16 loads in flight at 1 M weights).
+#ifndef RUDRA_MID_THREADS
+#define RUDRA_MID_THREADS 32
+#endif
+#ifndef RUDRA_MID_DEPTH
+#define RUDRA_MID_DEPTH 16
+#endif
+// Block size and loads in flight of the one-weight-per-thread kernel.
+#ifndef RUDRA_SMALL_THREADS
+#define RUDRA_SMALL_THREADS 128
+#endif
+#ifndef RUDRA_SMALL_DEPTH
+#define RUDRA_SMALL_DEPTH 8
+#endif
+
 // The per-weight rule.  Momentum SGD: u = acc + (sum s) wd theta; v' = m v + u; theta' = theta - v'.
 // AdaGrad: g = acc + wd theta (acc already the weighted mean gradient); h' = h + g^2;
 // theta' = theta - (sum s) g / (sqrt(h') + eps).
@@ -205,7 +221,7 @@ __global__ void __launch_bounds__(THREADS) update_kernel_small(const __grid_cons
 
 template <typename G, int OPT, bool STATE>
 cudaError_t launch_small(const UpdateParams& p, cudaStream_t stream) {
-  constexpr int THREADS = 128, DEPTH = 8;
+  constexpr int THREADS = RUDRA_SMALL_THREADS, DEPTH = RUDRA_SMALL_DEPTH;
   const uint64_t blocks = (p.n + THREADS - 1) / THREADS;
   update_kernel_small<G, OPT, STATE, DEPTH, THREADS><<<(unsigned)blocks, THREADS, 0, stream>>>(p);
   return cudaGetLastError();
@@ -247,7 +263,7 @@ cudaError_t launch_update(const UpdateParams& p, GradType gtype, Optim optim, in
   const bool small = p.n / kUnit < sms * 16 * 256;
   if (gtype == kBF16)
     return small ? launch_typed<__nv_bfloat16, 8, 64>(p, optim, stream) : launch_typed<__nv_bfloat16, 8, 256>(p, optim, stream);
-  return small ? launch_typed<float, 8, 64>(p, optim, stream) : launch_typed<float, 4, 256>(p, optim, stream);
+  return small ? launch_typed<float, RUDRA_MID_DEPTH, RUDRA_MID_THREADS>(p, optim, stream) : launch_typed<float, 4, 256>(p, optim, stream);
 }
 
 }  // namespace rudra

@@ -12,6 +12,9 @@
 struct OraEvent { int32_t kind; uint32_t learner; uint64_t pulled_ts, ts, seq, tick; };
 extern "C" {
 void* ora_sched_create(uint32_t, uint32_t, int32_t, uint64_t, double, int32_t);
+void* ora_sched_create_tree(uint32_t, uint32_t, int32_t, uint64_t, double, int32_t, uint32_t);
+int32_t ora_sched_on_pull(void*, uint32_t, uint64_t);
+int64_t ora_ps_push_relay(void*, const void* const*, const uint64_t*, uint32_t);
 void ora_sched_destroy(void*);
 void ora_sched_run(void*, uint64_t, OraEvent*);
 void* ora_ps_create(uint64_t, uint32_t, uint32_t, float, float, float);
@@ -50,6 +53,27 @@ int main() {
     }
   }
   if (rudra_sched_create(4, 5, 1, 0, 0.3, 0) != nullptr) return 4;
+  // learners -> leaves -> root, with one learner reporting the weights it really holds now and then
+  const struct { uint32_t lam, n; int mode; uint32_t fanin; } trees[] = {{12, 2, 1, 3}, {54, 18, 1, 3}, {8, 1, 0, 4}, {60, 4, 2, 5}, {6, 2, 2, 1}};
+  for (const auto& t : trees) {
+    rudra_sched* s = rudra_sched_create_tree(t.lam, t.n, t.mode, 7, 0.3, 0, t.fanin);
+    void* o = ora_sched_create_tree(t.lam, t.n, t.mode, 7, 0.3, 0, t.fanin);
+    if (!s || !o) return 11;
+    uint64_t held = 0;
+    for (int i = 0; i < 20000; ++i) {
+      rudra_event a;
+      OraEvent b;
+      if (rudra_sched_next(s, &a, 1) != 1) return 12;
+      ora_sched_run(o, 1, &b);
+      if (std::memcmp(&a, &b, sizeof(a)) != 0) return 13;
+      if (a.learner == 0 && (a.kind == RUDRA_EV_PULL || a.kind == RUDRA_EV_PULL_SKIP) && t.mode != 0) {
+        if (i % 3 == 0) held = a.ts;
+        else if (rudra_sched_on_pull(s, 0, held) != 0 || ora_sched_on_pull(o, 0, held) != 0) return 14;
+      }
+    }
+    rudra_sched_destroy(s);
+    ora_sched_destroy(o);
+  }
   // the oracle's update loop: every optimizer, policy, precision mode and gradient type, ragged sizes
   for (uint64_t N : {1ull, 7ull, 1000ull}) {
     for (int opt = 0; opt < 2; ++opt) for (int pol = 0; pol < 3; ++pol) for (int dt = 0; dt < 2; ++dt) for (int strict = 0; strict < 2; ++strict) {
@@ -70,8 +94,18 @@ int main() {
         }
         if (ora_ps_step(ps) != 1) return 7;
       }
+      // one more update through the server tree: a leaf's average of two, and a third gradient directly
+      {
+        const void* two[2] = {dt ? (const void*)g16.data() : (const void*)g32.data(), dt ? (const void*)g16.data() : (const void*)g32.data()};
+        const uint64_t stamps[2] = {5, 3};
+        if (ora_ps_push_relay(ps, two, stamps, 2) != 2) return 15;
+        if (ora_ps_push_relay(ps, two, stamps, 2) >= 0) return 16;   // would straddle two updates
+        if (ora_ps_push(ps, two[0], 4) != 3 || ora_ps_step(ps) != 1) return 17;
+        for (int l = 0; l < 3; ++l) ora_ps_push(ps, two[0], 6);
+        ora_ps_step(ps);
+      }
       if (ora_ps_push(ps, g32.data(), 99) >= 0) return 8;   // a gradient from the future
-      if (ora_ps_pull(ps, out.data()) != 5) return 9;
+      if (ora_ps_pull(ps, out.data()) != 7) return 9;
       if (!(out[N - 1] < 0.01f)) return 10;
       ora_ps_destroy(ps);
     }

@@ -23,7 +23,21 @@ int main(void) {
     if (ev[i].kind == RUDRA_EV_PUSH) { ++pushes; if (ev[i].pulled_ts > ev[i].ts) return 3; }
     if (ev[i].kind == RUDRA_EV_STEP) ++steps;
   }
+  if (rudra_sched_on_pull(s, 1, 0) != 0 || rudra_sched_on_pull(s, 99, 0) != RUDRA_E_INVAL) return 7;
+  if (rudra_sched_on_pull(s, 1, 1000000u) != RUDRA_E_BAD_TS) return 8;
   rudra_sched_destroy(s);
+  /* learners behind a server tree: 2 leaves of 3; a fan-in that does not divide c is refused */
+  s = rudra_sched_create_tree(6, 1, RUDRA_SCHED_SOFTSYNC_ROUNDS, 42u, 0.3, 0, 3);
+  if (!s || rudra_sched_next(s, ev, 64) != 64) return 9;
+  {
+    unsigned relays = 0;
+    for (i = 0; i < 64; ++i) relays += ev[i].kind == RUDRA_EV_RELAY;
+    if (relays < 8) return 10;
+  }
+  rudra_sched_destroy(s);
+  if (rudra_sched_create_tree(6, 2, RUDRA_SCHED_SOFTSYNC_ROUNDS, 42u, 0.3, 0, 2) != NULL) return 11;
+  if (rudra_leaf_average(NULL, 3, RUDRA_GRAD_F32, 64, NULL, NULL) != RUDRA_E_INVAL) return 12;
+  if (rudra_ps_push_group(NULL, NULL, 1, NULL, 1) != RUDRA_E_INVAL) return 13;
   /* bad arguments are refused before any device work, with a reason */
   if (rudra_ps_create(0, 4, 1, 0.1f, 0.0f, 0.0f) != NULL) return 4;
   if (rudra_ps_step(NULL) != RUDRA_E_INVAL) return 5;
