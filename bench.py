@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller vector; traffic grows in
 # proportion to the vector length).  Valid only for the kernel sources they were taken on.
 NCU_TRAFFIC = {
-    ("imagenet", 18): {"bytes_per_weight": 438.6, "kernel_sha": "e10c2a326020e428",
+    ("imagenet", 18): {"bytes_per_weight": 438.63, "kernel_sha": "02dea1760893a048",
                        "source": "profiles/update_kernel_imagenet_window18.md"},
 }
 
@@ -578,7 +578,8 @@ def run_ours(args, w):
         del extra, srcs, dsts
 
     e2e_ms, e2e_steps, h0, h1 = float('nan'), 0, None, None
-    if not args.kernel_only:
+    no_e2e = args.kernel_only or bool(args.tree)   # a leaf's relay has no host-buffer form: the tree is measured on the device
+    if not no_e2e:
         # end to end through the C interface with host buffers: gradients travel host -> device inside
         # the timed region and every pulled copy of the weights travels device -> host
         e2e_steps = min(args.steps, 16 if N > (1 << 24) else 200)
@@ -638,7 +639,7 @@ def run_ours(args, w):
         del bufs, slots
         torch.cuda.empty_cache()
         others = {}
-        for name, osteps, owarm in (("cifar10", 6000, 300), ("stress", 40, 4)):
+        for name, osteps, owarm in (("cifar10", 6000, 300), ("stress", 40, 4), ("imagenet72m", 180, 18)):
             ow = synth.WORKLOADS[name]
             orun = DeviceRun(rb, torch, ow, args, seed, stream)
             oW = default_window(ow)
@@ -665,7 +666,7 @@ def run_ours(args, w):
         # learners on this GPU, their averaging fused into the root's launch), and the leaf's own kernel
         k = 3
         trun = DeviceRun(rb, torch, w, args, seed, stream, fanin=k)
-        tsteps, twarm = min(args.steps, 360), W
+        tsteps, twarm = 360, W
         treg = timed_region(trun, w, make_windows(w, twarm + tsteps, fanin=k), twarm, tsteps, W, barrier)
         tbytes = sum(b["bytes_per_launch"] * b["launches"] for b in launch_shapes(w, N, W, treg).values())
         avg = torch.empty(N, dtype=torch.float32, device="cuda")
@@ -738,7 +739,7 @@ def run_ours(args, w):
             "one_message_at_a_time": single,
             "gpu_launches": launches,
             "clocks": clocks,
-            "e2e": None if args.kernel_only else {
+            "e2e": None if no_e2e else {
                 "value": replicas.whole_job_rate(e2e_steps, world, e2e_ms), "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": (h1["h2d_bytes"] - h0["h2d_bytes"]) // e2e_steps,
                 "d2h_bytes_per_step": (h1["d2h_bytes"] - h0["d2h_bytes"]) // e2e_steps,
@@ -835,7 +836,7 @@ def run_leaf_average(args, w):
 
     N, k = w.nparams, args.leaf_average
     g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
-    nbuf = max(k, min(54, int(6e9 // (N * g))) // k * k)
+    nbuf = max(k, (args.buffers or min(54, int(6e9 // (N * g)))) // k * k)
     bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype) for l in range(nbuf)]
     avg = torch.empty(N, dtype=torch.float32, device="cuda")
     stream = torch.cuda.Stream()
