@@ -34,31 +34,47 @@ UNIT = "updates/s"
 FALLBACK_HBM_GBS = 6650.0
 
 
-# DRAM traffic per weight of one launch of the dominant kernel, from ncu captures summarised under
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller vector; traffic grows in
-# proportion to the vector length).  Valid only for the kernel sources they were taken on.
+# DRAM traffic of one launch, from ncu captures summarised under profiles/ (dram__bytes_read.sum +
+# dram__bytes_write.sum).  The windowed update kernel was captured on a smaller vector with the same
+# launch shape (the full-size launch holds 26 GB of distinct buffers) and is scaled by the vector
+# length; the copy and leaf kernels were captured at full size.  Each record is valid only for the
+# kernel sources it was taken on.
 NCU_TRAFFIC = {
-    ("imagenet", 18): {"bytes_per_weight": 438.63, "kernel_sha": "02dea1760893a048",
-                       "source": "profiles/update_kernel_imagenet_window18.md"},
+    # (kernel, workload, updates, gradient vectors, weight copies)
+    ("update", "imagenet", 18, 54, 54): {"bytes_per_weight": 438.63, "sources": ("update.cu", "kernels.cuh", "vec.cuh"),
+                                         "sha": "02dea1760893a048", "source": "profiles/update_kernel_imagenet_window18.md"},
+    # (kernel, destinations)
+    ("snapshot", 1): {"bytes_per_launch_at": (60965224, 433.3e6), "sources": ("snapshot.cu", "kernels.cuh"),
+                      "sha": "4ac493055d27c19b", "source": "profiles/snapshot_kernel_imagenet_pull.md"},
+    # (kernel, fan-in, bytes per gradient element)
+    ("leaf", 3, 4): {"bytes_per_launch_at": (60965224, 926.8e6), "sources": ("leaf.cu", "kernels.cuh", "vec.cuh"),
+                     "sha": "2978ad1718fa79f8", "source": "profiles/leaf_average_kernel_imagenet_fanin3.md"},
 }
 
 
-def kernel_sources_sha():
+def sources_sha(files):
     import hashlib
 
     h = hashlib.sha256()
-    for f in ("update.cu", "kernels.cuh", "vec.cuh"):
+    for f in files:
         with open(os.path.join(ROOT, "paper_1509_04210_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
 
 
-def ncu_traffic(workload, window, nparams):
-    """Bytes per launch from the recorded capture, or None if there is none for this shape or the
-    kernel has changed since."""
-    rec = NCU_TRAFFIC.get((workload, window))
-    if rec is None or rec["kernel_sha"] != kernel_sources_sha():
+def kernel_sources_sha():
+    return sources_sha(("update.cu", "kernels.cuh", "vec.cuh"))
+
+
+def ncu_traffic(key, nparams):
+    """Bytes per launch from the recorded capture, or None if there is none for this kernel and
+    launch shape or the kernel's sources have changed since."""
+    rec = NCU_TRAFFIC.get(key)
+    if rec is None or rec["sha"] != sources_sha(rec["sources"]):
         return None
+    if "bytes_per_launch_at" in rec:
+        n, b = rec["bytes_per_launch_at"]
+        return float(b) if n == nparams else None
     return rec["bytes_per_weight"] * nparams
 
 
@@ -691,7 +707,8 @@ def run_ours(args, w):
                 "kernel": "leaf_average_kernel (a leaf's mean of its %d learners' gradients, one float vector out)" % k,
                 "bound": "hbm", "achieved": float(N) * (k * g + 4) / (leaf_us * 1e-6) / 1e9, "peak": peak_now, "unit": "GB/s",
                 "frac": float(N) * (k * g + 4) / (leaf_us * 1e-6) / 1e9 / peak_now, "launches_timed": reps,
-                "avg_launch_us": leaf_us, "bytes_per_launch": float(N) * (k * g + 4), "traffic": None},
+                "avg_launch_us": leaf_us, "bytes_per_launch": float(N) * (k * g + 4),
+                "traffic": ncu_traffic(("leaf", k, g), N)},
         }
         trun.close()
         del trun, avg
@@ -752,7 +769,8 @@ def run_ours(args, w):
                 "launch_us": None if not launch_ms else {
                     "min": 1e3 * min(launch_ms), "median": 1e3 * float(np.median(launch_ms)), "max": 1e3 * max(launch_ms)},
                 "frac_of_8TBs_datasheet": achieved / 8000.0,
-                "traffic": None if (W == 0 or not full) else ncu_traffic(w.name, full["updates"], N),
+                "traffic": None if (W == 0 or not full or views) else ncu_traffic(
+                    ("update", w.name, full["updates"], full["gradient_vectors"], full["weight_copies"]), N),
                 "mix_ceiling": mix,
                 "frac_of_mix_ceiling": None if not mix else achieved / mix["gbs"],
                 "other_launch_shapes": other_shapes,
@@ -763,7 +781,7 @@ def run_ours(args, w):
                 "bound": "hbm", "achieved": pull_roof["bytes"] / (pull_roof["us"] * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
                 "frac": pull_roof["bytes"] / (pull_roof["us"] * 1e-6) / 1e9 / peak, "peak_kind": "of %s" % peak_kind,
                 "launches_timed": pull_roof["launches"], "avg_launch_us": pull_roof["us"],
-                "bytes_per_launch": pull_roof["bytes"], "traffic": None,
+                "bytes_per_launch": pull_roof["bytes"], "traffic": ncu_traffic(("snapshot", pull_roof["ndst"]), N),
                 "where": "the one-message-at-a-time leg of this run: every pull a launch of its own",
             },
             "other_workloads": others,

@@ -567,6 +567,8 @@ int rudra_ps_set_option(rudra_ps* ps, int key, int64_t value) {
   return guarded([&]() -> int {
     if (!valid(ps)) return fail(RUDRA_E_INVAL, "bad handle");
     if (!ps->queue.empty()) return fail(RUDRA_E_STATE, "options can only change while no gradient is queued");
+    for (const auto& leaf : ps->leaf_pending)
+      if (!leaf.empty()) return fail(RUDRA_E_STATE, "options can only change while no leaf holds a gradient");
     DeviceScope dev(ps->device);
     switch (key) {
       case RUDRA_OPT_GRAD_DTYPE:
@@ -596,8 +598,6 @@ int rudra_ps_set_option(rudra_ps* ps, int key, int64_t value) {
       case RUDRA_OPT_TREE_FANIN:
         if (value < 0 || (value > 0 && (ps->lambda % value != 0 || ps->c % value != 0)))
           return fail(RUDRA_E_INVAL, "fan-in %lld must divide lambda = %u and c = %u", (long long)value, ps->lambda, ps->c);
-        for (const auto& leaf : ps->leaf_pending)
-          if (!leaf.empty()) return fail(RUDRA_E_STATE, "leaves still hold gradients");
         ps->fanin = (uint32_t)value;
         ps->leaf_pending.assign(value ? ps->lambda / (uint32_t)value : 0, {});
         return 0;
