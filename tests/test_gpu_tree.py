@@ -364,3 +364,75 @@ def test_copy_push_mode_lets_the_caller_overwrite_its_buffer(N):
     np.testing.assert_array_equal(tha, thb)
     np.testing.assert_array_equal(sta, stb)
     a.close(), b.close()
+
+
+@pytest.mark.parametrize("N", [1, 5, 8, 4099])
+def test_widest_tree_group_fills_the_launch_table(N):
+    """lambda = 128, n = 1: one update of c = 128 gradients (the table's limit) as two leaves of 64,
+    once as raw vectors and once as relayed averages, on vectors shorter than one 256-bit unit too."""
+    import torch
+
+    lam, k = 128, 64
+    for relayed in (False, True):
+        rb, gpu, cpus = _pair(N, lam, 1, ora.LR_PER_GRADIENT, ora.OPT_MOMENTUM_SGD, 0.9, 5e-4)
+        cpu = cpus[0]
+        for upd in range(2):
+            ts = gpu.timestamp()
+            keep = []
+            for leaf in range(2):
+                gs = [_grad(N, leaf * k + i, upd, synth.GRAD_F32) for i in range(k)]
+                stamps = [max(0, ts - (i % 2)) for i in range(k)]
+                dev = [to_device(g) for g in gs]
+                keep.append(dev)
+                if relayed:
+                    avg = torch.empty(N, device="cuda")
+                    keep.append(avg)
+                    rb.leaf_average(dev, synth.GRAD_F32, N, avg)
+                    gpu.push_group([avg], stamps)
+                else:
+                    gpu.push_group(dev, stamps)
+                cpu.push_relay(gs, stamps)
+            assert gpu.step() == 1 and cpu.step() == 1
+            gpu.sync()
+            _check_integers(gpu, cpu)
+            th, st = _state(gpu, N)
+            tol = REL_ONE_STEP if upd == 0 else REL_100_STEPS
+            assert rel_err(th, cpu.pull()[0]) <= tol and rel_err(st, cpu.state()) <= tol
+        gpu.close()
+
+
+def test_empty_batches_and_partial_leaves_carry_over():
+    """run_events with no events does nothing; a leaf left half full at the end of a batch is
+    completed by the next batch; options cannot change while a leaf holds a gradient."""
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    N, lam, n, k = 3001, 8, 2, 2
+    rb, gpu, cpus = _pair(N, lam, n, ora.LR_PAPER_N, ora.OPT_MOMENTUM_SGD, 0.9, 5e-4)
+    cpu = cpus[0]
+    gpu.set_option(rb.OPT_TREE_FANIN, k)
+    grads_np = [_grad(N, l, 0, synth.GRAD_F32) for l in range(lam)]
+    grads = [to_device(g) for g in grads_np]
+    slots = [torch.empty(N, device="cuda") for _ in range(lam)]
+    ev = rb.Scheduler(lam, n, rb.SCHED_SOFTSYNC_ROUNDS, 3, 0.3, False, k).next(200)
+    assert gpu.run_events(ev[:0], grads, slots) == 0 and gpu.timestamp() == 0
+    first_push = int(np.flatnonzero(ev["kind"] == rb.EV_PUSH)[0])
+    assert gpu.run_events(ev[: first_push + 1], grads, slots) == 0          # one gradient sits at its leaf
+    with pytest.raises(rb.RudraError) as e:
+        gpu.set_option(rb.OPT_LR_POLICY, rb.LR_GROUP_MEAN)
+    assert e.value.code == rb.E_STATE
+    done = gpu.run_events(ev[first_push + 1:], grads, slots)
+    at_leaf = {}
+    for e in ev:
+        kind, l = int(e["kind"]), int(e["learner"])
+        if kind == ora.PUSH:
+            at_leaf.setdefault(l // k, []).append((grads_np[l], int(e["pulled_ts"])))
+        elif kind == ora.RELAY:
+            msg = at_leaf.pop(l)
+            cpu.push_relay([g for g, _ in msg], [p for _, p in msg])
+        elif kind == ora.STEP:
+            assert cpu.step() == 1
+    assert done == cpu.timestamp() == gpu.timestamp() > 10
+    th, st = _state(gpu, N)
+    assert rel_err(th, cpu.pull()[0]) <= REL_100_STEPS and rel_err(st, cpu.state()) <= REL_100_STEPS
+    gpu.close()
