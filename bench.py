@@ -528,10 +528,32 @@ def run_ours(args, w):
     ps, bufs, slots, nbufs = run.ps, run.bufs, run.slots, run.nbufs
     warm_done = args.warmup if W == 0 else -(-args.warmup // W) * W
     extra_steps = 0 if (W == 0 or views or args.tree) else min(args.steps, 216)
-    windows = make_windows(w, warm_done + args.steps + extra_steps, fanin=args.tree)
-    extra_windows = windows[warm_done + args.steps:]
+    # a short timed region holds few full-window launches: after it, finish the learners' round and
+    # time ten more full backlogs, reported beside the roofline (not part of `value`)
+    more = 10 if (W >= 1 and args.steps // max(W, 1) < 10) else 0
+    tail = (-args.steps) % W if more else 0
+    windows = make_windows(w, warm_done + args.steps + tail + more * W + extra_steps, fanin=args.tree)
+    extra_windows = windows[warm_done + args.steps + tail + more * W:]
     region = timed_region(run, w, windows, args.warmup, args.steps, W, barrier,
                           lambda: ClockSampler(visible_gpu_index(local_rank)))
+    more_launches = None
+    if more:
+        at = warm_done + args.steps
+        if tail:
+            run.backlog(np.concatenate(windows[at: at + tail]), W, [], [])
+        run.events(more + 2)
+        mev, mbytes = [], []
+        gb = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
+        for i in range(more):
+            chunk = np.concatenate(windows[at + tail + i * W: at + tail + (i + 1) * W])
+            _, vectors, ncopies = batch_shape(w, chunk)
+            mbytes.append(float(N) * (vectors * gb + state_bytes(w) + 4 * ncopies))
+            run.backlog(chunk, W, mev, [])
+        torch.cuda.synchronize()
+        mus = [1e3 * a.elapsed_time(b) for a, b in mev]
+        more_launches = {"launches": more, "avg_launch_us": float(np.mean(mus)), "min": min(mus), "max": max(mus),
+                         "bytes_per_launch": float(np.mean(mbytes)),
+                         "gbs": float(np.sum(mbytes)) / (float(np.sum(mus)) * 1e-6) / 1e9}
     ms, launch_ms, clocks = region["ms"], region["launch_ms"], region["clocks"]
     kern_ms = float(sum(launch_ms))
     launches, pulls, copies = region["launches"], region["pulls"], region["copies"]
@@ -774,6 +796,9 @@ def run_ours(args, w):
                 "mix_ceiling": mix,
                 "frac_of_mix_ceiling": None if not mix else achieved / mix["gbs"],
                 "other_launch_shapes": other_shapes,
+                "more_full_window_launches": None if not more_launches or views else dict(
+                    more_launches,
+                    note="the same server right after the timed region, the round finished first; not part of value"),
             },
             "roofline_pull": None if not pull_roof else {
                 "kernel": "snapshot_kernel (pullWeights: one read of the weights, %d written cop%s)" % (
