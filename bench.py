@@ -482,8 +482,8 @@ def launch_shapes(w, N, W, region):
     for (updates, vectors, copies), ms in zip(region["shapes"], region["launch_ms"]):
         if region.get("views"):   # shared versions: a version is written once however many learners take it
             copies = region["copies"] * updates / total_updates
-        rec = out.setdefault(updates, {"updates": updates, "gradient_vectors": vectors, "weight_copies": copies, "launches": 0,
-                                       "ms": 0.0})
+        rec = out.setdefault((updates, vectors, copies), {"updates": updates, "gradient_vectors": vectors,
+                                                          "weight_copies": copies, "launches": 0, "ms": 0.0})
         rec["launches"] += 1
         rec["ms"] += ms
         rec["bytes_per_launch"] = float(N) * (vectors * g + sb + 4 * copies + 4 * extra_per_call)
@@ -586,7 +586,11 @@ def run_ours(args, w):
                          "bytes": float(N) * (4 + 4 * ndst)}
 
     shapes = launch_shapes(w, N, W, region) if W != 0 else {}
-    full = shapes.get(W) or (shapes[max(shapes)] if shapes else None)
+    # the launch shape the roofline describes: the full window (W updates) seen most often, else the largest seen
+    full = None
+    if shapes:
+        whole = [b for b in shapes.values() if b["updates"] == W]
+        full = max(whole, key=lambda b: b["launches"]) if whole else shapes[max(shapes)]
 
     # What HBM delivers on this GPU, in this run, for the same mix of reads and writes as one
     # full-window launch of the dominant kernel: a probe kernel that only streams that many vectors
