@@ -722,10 +722,47 @@ def run_ours(args, w):
         l1.record(stream)
         torch.cuda.synchronize()
         leaf_us = 1e3 * l0.elapsed_time(l1) / reps
+        # the other form of the relay, one message at a time: every leaf runs its averaging kernel and
+        # the root receives one float vector per leaf (what crosses the link when leaves sit on other GPUs)
+        mrun = DeviceRun(rb, torch, w, args, seed, stream)
+        mwin = make_windows(w, 2 * W + 108, fanin=k)
+        avgs = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(w.lam // k)]
+        held = {}
+
+        def relay_window(win):
+            for kind, learner, pulled_ts in zip(win["kind"].tolist(), win["learner"].tolist(), win["pulled_ts"].tolist()):
+                if kind == EV_PUSH:
+                    held.setdefault(learner // k, []).append((mrun.bufs[learner], pulled_ts))
+                elif kind == 6:   # RELAY
+                    msg = held.pop(learner)
+                    rb.leaf_average([b for b, _ in msg], w.grad_dtype, N, avgs[learner], stream)
+                    mrun.ps.push_group([avgs[learner]], [p for _, p in msg])
+                elif kind == EV_STEP:
+                    mrun.ps.step()
+                elif kind == EV_PULL:
+                    mrun.ps.pull(mrun.slots[learner])
+
+        for win in mwin[: 2 * W]:
+            relay_window(win)
+        barrier()
+        m0, m1 = mrun.pair()
+        m0.record(stream)
+        for win in mwin[2 * W:]:
+            relay_window(win)
+        m1.record(stream)
+        barrier()
+        relay_rate = 108 / (m0.elapsed_time(m1) * 1e-3)
+        mrun.close()
+        del mrun, avgs
+        torch.cuda.empty_cache()
         peak_now = measured_hbm_peak()[0]
         others["imagenet_tree_fanin3"] = {
             "value": tsteps / (treg["ms"] * 1e-3), "unit": UNIT, "steps": tsteps, "window": W, "fanin": k,
             "relay": "leaves share the root's GPU: raw gradients handed over, averaged inside the update kernel",
+            "materialised_relay_one_message_at_a_time": {
+                "value": relay_rate, "unit": UNIT, "steps": 108,
+                "how": "every leaf runs rudra_leaf_average, the root takes one float vector per leaf "
+                       "(rudra_ps_push_group), step and pull as separate calls; compare one_message_at_a_time"},
             "bytes_per_param_per_step": tbytes / N / tsteps, "hbm_gbs": tbytes / (treg["ms"] * 1e-3) / 1e9,
             "gpu_launches": treg["launches"], "avg_launch_us": 1e3 * float(np.mean(treg["launch_ms"])),
             "host_us_per_call": float(np.median(treg["host_us"])),
