@@ -414,15 +414,18 @@ class DeviceRun:
                     e1.record(stream)
                     pull_events.append((e0, e1, len(slots)))
 
-    def backlog(self, chunk, W, timed, host_s):
-        """A backlog of update windows through one rudra_ps_run_events call."""
-        e0, e1 = self.pair()
-        e0.record(self.stream)
+    def backlog(self, chunk, W, timed, host_s, with_events=True, address=None):
+        """A backlog of update windows through one rudra_ps_run_events call (chunk: a contiguous event
+        array that the caller keeps alive).  with_events: bracket the call with two timing events."""
+        if with_events:
+            e0, e1 = self.pair()
+            e0.record(self.stream)
         t0 = time.perf_counter()
-        self.ps.run_events(chunk, self.gtable, self.stable, W)
+        self.ps.run_events_at(address or chunk.ctypes.data, len(chunk), self.gtable, self.stable, W)
         host_s.append(time.perf_counter() - t0)
-        e1.record(self.stream)
-        timed.append((e0, e1))
+        if with_events:
+            e1.record(self.stream)
+            timed.append((e0, e1))
 
     def close(self):
         self.ps.close()
@@ -432,7 +435,10 @@ class DeviceRun:
 def timed_region(run, w, windows, warmup, steps, W, barrier, sampler_factory=None):
     """Warm-up, then exactly ``steps`` update windows between two events.  With a backlog size W the
     warm-up is rounded up to whole backlogs so that the timed backlogs start where a round of the
-    learners starts; the timed windows are handed over as backlogs of W (the last may be shorter)."""
+    learners starts; the timed windows are handed over as backlogs of W (the last may be shorter).
+    Every launch is bracketed by timing events when the workload streams from HBM (the roofline is
+    formed from those); for L2-resident, launch-bound workloads only every eighth call is, so that
+    the event records do not slow the host loop that is the bottleneck there."""
     torch, stream, ps = run.torch, run.stream, run.ps
     warm = warmup if W == 0 else -(-warmup // W) * W
     wins = windows[: warm + steps]
@@ -442,7 +448,10 @@ def timed_region(run, w, windows, warmup, steps, W, barrier, sampler_factory=Non
     else:
         warm_batches = [np.concatenate(wins[i:i + W]) for i in range(0, warm, W)]
         batches = [np.concatenate(wins[i:i + W]) for i in range(warm, warm + steps, W)]
-    shapes = [batch_shape(w, b) for b in batches]
+    stride = 1 if (W == 0 or w.nparams * 8 > 126e6) else 8
+    all_shapes = [batch_shape(w, b) for b in batches]
+    shapes = all_shapes[::stride]
+    addresses = [None] * len(batches) if W == 0 else [b.ctypes.data for b in batches]
     junk, host_s = [], []
     for b in warm_batches:
         run.messages(b, junk) if W == 0 else run.backlog(b, W, junk, [])
@@ -456,8 +465,8 @@ def timed_region(run, w, windows, warmup, steps, W, barrier, sampler_factory=Non
     start, end = run.pair()
     timed = []
     start.record(stream)
-    for b in batches:
-        run.messages(b, timed) if W == 0 else run.backlog(b, W, timed, host_s)
+    for i, b in enumerate(batches):
+        run.messages(b, timed) if W == 0 else run.backlog(b, W, timed, host_s, i % stride == 0, addresses[i])
     end.record(stream)
     barrier()
     clocks = sampler.stop() if sampler else None
@@ -467,7 +476,17 @@ def timed_region(run, w, windows, warmup, steps, W, barrier, sampler_factory=Non
         "host_us": [1e6 * t for t in host_s], "warmup_done": warm, "clocks": clocks,
         "launches": c1["launches"] - c0["launches"], "pulls": c1["pulls"] - c0["pulls"],
         "copies": c1["weight_copies"] - c0["weight_copies"], "batches": len(batches), "views": run.views,
+        "launches_sampled_every": stride, "all_shapes": all_shapes,
     }
+
+
+def path_bytes_of(w, N, region):
+    """Algorithmic bytes of everything the timed region's run_events calls asked for."""
+    g = 2 if w.grad_dtype == synth.GRAD_BF16 else 4
+    extra = max(0, region["launches"] - region["batches"])          # copy launches split off: one more read of the weights each
+    vectors = sum(v for _, v, _ in region["all_shapes"])
+    copies = region["copies"] if region.get("views") else sum(c for _, _, c in region["all_shapes"])
+    return float(N) * (vectors * g + state_bytes(w) * region["batches"] + 4 * copies + 4 * extra)
 
 
 def launch_shapes(w, N, W, region):
@@ -689,7 +708,7 @@ def run_ours(args, w):
             reg = timed_region(orun, ow, owin, owarm, osteps, oW, barrier)
             og = 2 if ow.grad_dtype == synth.GRAD_BF16 else 4
             osb = 16 if ow.momentum else 8
-            obytes = sum(b["bytes_per_launch"] * b["launches"] for b in launch_shapes(ow, ow.nparams, oW, reg).values())
+            obytes = path_bytes_of(ow, ow.nparams, reg)
             others[name] = {
                 "value": osteps / (reg["ms"] * 1e-3), "unit": UNIT, "steps": osteps, "warmup": reg["warmup_done"],
                 "nparams": ow.nparams, "lambda": ow.lam, "n": ow.n, "c": ow.c,
@@ -710,7 +729,7 @@ def run_ours(args, w):
         trun = DeviceRun(rb, torch, w, args, seed, stream, fanin=k)
         tsteps, twarm = 360, W
         treg = timed_region(trun, w, make_windows(w, twarm + tsteps, fanin=k), twarm, tsteps, W, barrier)
-        tbytes = sum(b["bytes_per_launch"] * b["launches"] for b in launch_shapes(w, N, W, treg).values())
+        tbytes = path_bytes_of(w, N, treg)
         avg = torch.empty(N, dtype=torch.float32, device="cuda")
         for i in range(3):
             rb.leaf_average(trun.bufs[3 * i: 3 * i + k], w.grad_dtype, N, avg, stream)
@@ -787,7 +806,7 @@ def run_ours(args, w):
             roof_launches, roof_us, roof_bytes = len(launch_ms), 1e3 * kern_ms / max(len(launch_ms), 1), kern_bytes / max(len(launch_ms), 1)
             label = "update_kernel (fused sumGradients + applyUpdate), one update per launch"
         else:
-            path_bytes = sum(b["bytes_per_launch"] * b["launches"] for b in shapes.values())
+            path_bytes = path_bytes_of(w, N, region)
             achieved, roof_launches, roof_us, roof_bytes = full["gbs"], full["launches"], full["avg_launch_us"], full["bytes_per_launch"]
             label = "update_kernel (fused sumGradients + applyUpdate), %d-update window with its %d pulls%s" % (
                 full["updates"], full["weight_copies"],
@@ -797,6 +816,7 @@ def run_ours(args, w):
         cfg["parallelism"] = "replicas x%d (one independent server per GPU)" % world
         cfg["window"] = W
         cfg["warmup_done"] = region["warmup_done"]
+        cfg["launches_timed_every"] = region["launches_sampled_every"]
         cfg["pull"] = ("zero-copy: learners share a pointer to the version they pulled (rudra_ps_enable_views)" if views
                        else "copy into each learner's slot")
         cfg["window_note"] = ("messages handled one at a time (push / step / pull)" if W == 0 else

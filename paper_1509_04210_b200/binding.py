@@ -259,6 +259,14 @@ class ParameterServer:
         sl = None if slots_dev is None else (slots_dev if isinstance(slots_dev, C.Array) else _ptr_array(slots_dev))
         return _check(lib().rudra_ps_run_events(self._h, ev.ctypes.data, len(ev), g, sl, int(max_window)))
 
+    def run_events_at(self, events_address, count, grads_table, slots_table, max_window=0):
+        """The same call for a caller that has marshalled its arguments once: the address of a
+        contiguous EVENT_DTYPE array that it keeps alive, and pointer tables from ``pointer_table``."""
+        code = _lib.rudra_ps_run_events(self._h, events_address, count, grads_table, slots_table, max_window)
+        if code < 0:
+            raise RudraError(code, last_error())
+        return code
+
     def timestamp(self):
         return _check(lib().rudra_ps_timestamp(self._h))
 

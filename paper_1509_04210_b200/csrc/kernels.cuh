@@ -12,6 +12,7 @@ enum GradType : int { kF32 = 0, kBF16 = 1 };
 enum Optim : int { kMomentumSgd = 0, kAdagrad = 1 };
 
 constexpr int kMaxWindow = 32;   // most updates one launch can carry
+constexpr uint8_t kNotLast = 0xFF;
 
 // Everything one launch of the fused kernel needs: a window of nupd consecutive updates (each
 // sumGradients + applyUpdate over c gradients) with the pulls that fall between them.  Passed by
@@ -30,6 +31,9 @@ struct UpdateParams {
   float abar[kMaxWindow];        // per update, AdaGrad: sum(s), the group's learning rate
   uint8_t dst_end[kMaxWindow + 1];
   uint8_t grad_end[kMaxWindow + 2];   // grad_end[0] = 0; one spare entry, read but never used, after the last update
+  // Filled by launch_update for the one-weight-per-thread kernel: per vector, kNotLast if it is not
+  // the last vector of its update, else the number of pull destinations served after that update.
+  uint8_t after[kMaxGroup];
   float* theta;
   float* state;                  // velocity (momentum SGD) or sum of squared gradients (AdaGrad)
   uint64_t n;                    // number of weights

@@ -187,31 +187,37 @@ __global__ void __launch_bounds__(THREADS) update_kernel(const __grid_constant__
 // its order are those of the kernel above.
 template <typename G, int OPT, bool STATE, int DEPTH, int THREADS>
 __global__ void __launch_bounds__(THREADS) update_kernel_small(const __grid_constant__ UpdateParams p) {
-  const uint64_t k = (uint64_t)blockIdx.x * THREADS + threadIdx.x;
-  if (k >= p.n) return;
+  const uint32_t k = blockIdx.x * THREADS + threadIdx.x;   // fewer than 2^18 weights: 32-bit indexing
+  if (k >= (uint32_t)p.n) return;
   float th = p.theta[k];
   float st = STATE ? p.state[k] : 0.f;
   uint32_t d = 0;
   for (const uint32_t d1 = p.dst_end[0]; d < d1; ++d) p.dst[d][k] = th;
-  const uint32_t total = p.grad_end[p.nupd];
-  uint32_t w = 0, last = p.grad_end[1];
+  // The vector table is padded to a whole number of chunks (launch_small), so neither the loads nor
+  // the fma chain need bounds checks; what a padding entry adds to acc after the last update is
+  // never used.
+  const uint32_t padded = (p.grad_end[p.nupd] + DEPTH - 1) / DEPTH * DEPTH;
+  uint32_t w = 0;
   float acc = 0.f;
-  for (uint32_t l0 = 0; l0 < total; l0 += DEPTH) {
-    float g[DEPTH];
-#pragma unroll
-    for (int i = 0; i < DEPTH; ++i)
-      if (l0 + i < total) g[i] = GradUnit<G>::scalar(p.grad[l0 + i], k);
+  for (uint32_t l0 = 0; l0 < padded; l0 += DEPTH) {
+    // the chunk's table entries are fetched together with its gradients, ahead of the dependent chain
+    float g[DEPTH], s[DEPTH];
+    uint32_t after[DEPTH];
 #pragma unroll
     for (int i = 0; i < DEPTH; ++i) {
-      if (l0 + i < total) {
-        acc = fmaf(p.scale[l0 + i], g[i], acc);
-        if (l0 + i + 1 == last) {
-          apply<OPT, STATE>(p, p.awd[w], p.abar[w], acc, th, st);
-          acc = 0.f;
-          ++w;
-          last = p.grad_end[w + 1];
-          for (const uint32_t d1 = p.dst_end[w]; d < d1; ++d) p.dst[d][k] = th;
-        }
+      g[i] = GradUnit<G>::scalar(p.grad[l0 + i], k);
+      s[i] = p.scale[l0 + i];
+      after[i] = p.after[l0 + i];
+    }
+#pragma unroll
+    for (int i = 0; i < DEPTH; ++i) {
+      acc = fmaf(s[i], g[i], acc);
+      const uint32_t pulls = after[i];
+      if (pulls != kNotLast) {   // last vector of update w: applyUpdate, then the pulls that follow it
+        apply<OPT, STATE>(p, p.awd[w], p.abar[w], acc, th, st);
+        acc = 0.f;
+        ++w;
+        for (const uint32_t d1 = d + pulls; d < d1; ++d) p.dst[d][k] = th;
       }
     }
   }
@@ -220,8 +226,17 @@ __global__ void __launch_bounds__(THREADS) update_kernel_small(const __grid_cons
 }
 
 template <typename G, int OPT, bool STATE>
-cudaError_t launch_small(const UpdateParams& p, cudaStream_t stream) {
+cudaError_t launch_small(const UpdateParams& window, cudaStream_t stream) {
   constexpr int THREADS = RUDRA_SMALL_THREADS, DEPTH = RUDRA_SMALL_DEPTH;
+  static_assert(kMaxGroup % DEPTH == 0, "the padded vector table must fit");
+  UpdateParams p = window;
+  const uint32_t total = p.grad_end[p.nupd];
+  for (uint32_t l = 0; l < (uint32_t)kMaxGroup; ++l) p.after[l] = kNotLast;
+  for (uint32_t u = 0; u < p.nupd; ++u) p.after[p.grad_end[u + 1] - 1] = (uint8_t)(p.dst_end[u + 1] - p.dst_end[u]);
+  for (uint32_t l = total; l % DEPTH != 0; ++l) {   // padding: a readable vector, no effect
+    p.grad[l] = p.grad[0];
+    p.scale[l] = 0.f;
+  }
   const uint64_t blocks = (p.n + THREADS - 1) / THREADS;
   update_kernel_small<G, OPT, STATE, DEPTH, THREADS><<<(unsigned)blocks, THREADS, 0, stream>>>(p);
   return cudaGetLastError();
