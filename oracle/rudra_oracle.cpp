@@ -14,15 +14,17 @@
 // Parity status of the parts the paper does not write out:
 //   * momentum / weight-decay form         : parity unpinned by the paper
 //     (the paper names "momentum 0.9" and a "weight regularization penalty"
-//     in Section 4.2 but prints no formula); pinned only by closed forms of
-//     the reading stated at OraclePS::step below.
+//     in Section 4.2 but prints no formula); the reading stated at
+//     OraclePS::step below is pinned by closed forms and, at a constant rate,
+//     by the trajectory of a library optimizer (torch.optim.SGD in float64).
 //   * sigma = 0 floor in the per-gradient and group-mean rate policies
 //     (alpha0/sigma is undefined at sigma = 0)  : parity unpinned by the paper.
 //   * AdaGrad form (Section 5.5 names the method, prints no formula)
 //                                           : parity unpinned by the paper; the
 //     reading at OraclePS::step is pinned by the direction of the first step
 //     (the sign of gradient plus penalty), by a decay-only scalar recurrence
-//     and by brute force in decimal arithmetic with unequal per-gradient rates.
+//     and by brute force in decimal arithmetic with unequal per-gradient rates,
+//     and at a constant rate by torch.optim.Adagrad's trajectory in float64.
 //   * Rudra-adv's server tree (Section 3.3 says that a leaf averages its
 //     learners' gradients and relays the average to its parent, and that the
 //     root applies the update; it does not say when a leaf relays, which
