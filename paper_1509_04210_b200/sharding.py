@@ -35,6 +35,10 @@ class ShardedServer:
     ``empty(n, kind)`` allocates a local vector of n elements for gradients (kind "grad") or weights
     (kind "weights") on the rank's device; tensors are torch tensors on that device.
     Every rank must make the same calls in the same order (they come from the same event stream).
+    On GPUs the slice copies and the collectives run on torch's current stream while the local
+    server enqueues on its own: leave the server on the default stream, or give it torch's current
+    stream (``set_stream``), so that a slice is complete before the update reads it and a pulled
+    range is complete before it is broadcast.
     """
 
     def __init__(self, make_server, nparams, c, empty, group=None):

@@ -1,7 +1,9 @@
-"""The two 60 965 224-weight workloads at their full stated lengths, in the launch configuration
-the benchmark times (one distinct gradient buffer and one slot per learner, backlogs handed to
-rudra_ps_run_events), against the CPU oracle: a sample of the weights over the whole run (exact,
-because weights never interact) and the whole vector over the first updates."""
+"""The workloads at their full stated sizes and lengths, in the launch configuration the benchmark
+times (one distinct gradient buffer and one slot per learner, backlogs handed to
+rudra_ps_run_events), against the CPU oracle: for the two 60 965 224-weight workloads a sample of
+the weights over the whole run (exact, because weights never interact) and the whole vector over
+the first updates; for the 1 M-weight workload a sample over its 2 000 updates; for the
+CIFAR10-scale workload every weight over its 10 000 updates."""
 import numpy as np
 import pytest
 
@@ -49,12 +51,14 @@ def _batches(rb, sched, w, updates, per_batch, cuts):
     return out
 
 
-def _run_full_size(w, updates, per_batch, max_window, checkpoints, seed):
+def _run_full_size(w, updates, per_batch, max_window, checkpoints, seed, strict=False, whole=False):
+    """strict: the oracle evaluates in fp32, one fused multiply-add per term, and the comparison is
+    bit for bit.  whole: every weight is compared instead of a sample."""
     import torch
     from paper_1509_04210_b200 import binding as rb
 
     N = w.nparams
-    idx = _sample_indices(N, 20000, seed)
+    idx = np.arange(N) if whole else _sample_indices(N, 20000, seed)
     idx_d = torch.from_numpy(idx).cuda()
     bufs = [synth.device_gradient(N, l, w.grad_std, w.grad_dtype) for l in range(w.lam)]
     slots = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(w.lam)]
@@ -64,6 +68,7 @@ def _run_full_size(w, updates, per_batch, max_window, checkpoints, seed):
     ps.set_weights(th0)
     o = ora.OraclePS(len(idx), w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
     o.set_grad_dtype(w.grad_dtype)
+    o.set_strict(strict)
     o.set_weights(to_host(th0[idx_d]))
     samples = [_host_view(b[idx_d], w) for b in bufs]
     gtable, stable = rb.pointer_table(bufs), rb.pointer_table(slots)
@@ -93,7 +98,7 @@ def _run_full_size(w, updates, per_batch, max_window, checkpoints, seed):
         if done in checkpoints or done == updates:
             ps.export_state(th, st)
             ps.sync()
-            tol = REL_ONE_STEP if done == 1 else REL_100_STEPS
+            tol = 0.0 if strict else REL_ONE_STEP if done == 1 else REL_100_STEPS
             e_th = rel_err(to_host(th[idx_d]), o.pull()[0])
             e_st = rel_err(to_host(st[idx_d]), o.state())
             assert e_th <= tol and e_st <= tol, (done, e_th, e_st)
@@ -101,7 +106,7 @@ def _run_full_size(w, updates, per_batch, max_window, checkpoints, seed):
     assert done == updates
     ps.sync()
     for l, want in slot_want.items():                         # each learner's copy: what the oracle handed it last
-        assert rel_err(to_host(slots[l][idx_d]), want) <= REL_100_STEPS, l
+        assert rel_err(to_host(slots[l][idx_d]), want) <= (0.0 if strict else REL_100_STEPS), l
     launches = ps.counters()["launches"]
     ps.close()
     return errs, launches
@@ -124,6 +129,29 @@ def test_stress_100_updates_with_their_broadcasts_at_full_size():
     errs, launches = _run_full_size(w, 100, 1, 1, {1, 2, 50}, seed=6)
     assert set(errs) >= {1, 100}
     assert launches == 200                                      # update + 128-way copy per window
+
+
+@pytest.mark.parametrize("strict", [False, True])
+def test_cifar10_10000_updates_every_weight(strict):
+    # 89 578 weights, lambda = n = 30 (c = 1, the staleness of Fig. 3b), momentum 0.9, decay 4e-3, 10 000
+    # updates in backlogs of one round (30 updates and their 30 pulls); the 1e-4 bar, stated for 100
+    # updates, is held to the end, and the fp32 evaluation of the oracle is matched bit for bit throughout
+    w = synth.WORKLOADS["cifar10"]
+    assert w.updates == 10000 and w.nparams == 89578
+    errs, launches = _run_full_size(w, 10000, 30, 0, {1, 100, 1000, 5000}, seed=7, strict=strict, whole=True)
+    assert set(errs) >= {1, 100, 10000}
+    assert launches <= 2 + (10000 + 29) // 30 + 4
+
+
+def test_mid_2000_updates_with_timed_learners():
+    # 1 M weights, lambda = 60, n = 4 (c = 15), learners with lognormal(0, 0.3) compute times, 2 000 updates in
+    # backlogs of 4 updates as the benchmark hands them over
+    w = synth.WORKLOADS["mid"]
+    assert w.updates == 2000 and w.nparams == 1000000
+    errs, _ = _run_full_size(w, 2000, 4, 0, {1, 100, 1000}, seed=8)
+    assert set(errs) >= {1, 100, 2000}
+    errs, _ = _run_full_size(w, 200, 4, 0, {1, 100}, seed=9, strict=True)
+    assert errs[200] == (0.0, 0.0)
 
 
 def test_imagenet_whole_vector_against_the_full_size_oracle():
