@@ -41,14 +41,14 @@ FALLBACK_HBM_GBS = 6650.0
 # kernel sources it was taken on.
 NCU_TRAFFIC = {
     # (kernel, workload, updates, gradient vectors, weight copies)
-    ("update", "imagenet", 18, 54, 54): {"bytes_per_weight": 438.63, "sources": ("update.cu", "kernels.cuh", "vec.cuh"),
-                                         "sha": "02dea1760893a048", "source": "profiles/update_kernel_imagenet_window18.md"},
+    ("update", "imagenet", 18, 54, 54): {"bytes_per_weight": 438.71, "sources": ("update.cu", "kernels.cuh", "vec.cuh"),
+                                         "sha": "9bd3787d26f56bbe", "source": "profiles/update_kernel_imagenet_window18.md"},
     # (kernel, destinations)
-    ("snapshot", 1): {"bytes_per_launch_at": (60965224, 433.3e6), "sources": ("snapshot.cu", "kernels.cuh"),
-                      "sha": "4ac493055d27c19b", "source": "profiles/snapshot_kernel_imagenet_pull.md"},
+    ("snapshot", 1): {"bytes_per_launch_at": (60965224, 433.7e6), "sources": ("snapshot.cu", "kernels.cuh"),
+                      "sha": "a821be77c12fccc9", "source": "profiles/snapshot_kernel_imagenet_pull.md"},
     # (kernel, fan-in, bytes per gradient element)
-    ("leaf", 3, 4): {"bytes_per_launch_at": (60965224, 926.8e6), "sources": ("leaf.cu", "kernels.cuh", "vec.cuh"),
-                     "sha": "2978ad1718fa79f8", "source": "profiles/leaf_average_kernel_imagenet_fanin3.md"},
+    ("leaf", 3, 4): {"bytes_per_launch_at": (60965224, 926.5e6), "sources": ("leaf.cu", "kernels.cuh", "vec.cuh"),
+                     "sha": "aac70d5e74ad45de", "source": "profiles/leaf_average_kernel_imagenet_fanin3.md"},
 }
 
 
