@@ -323,6 +323,35 @@ def workload_config(w):
 # ---------------------------------------------------------------------------------------------
 # the CUDA arm
 # ---------------------------------------------------------------------------------------------
+def link_probe(torch, pinned_src, pinned_dst, reps=6):
+    """GB/s per direction of plain pinned-memory copies over the host link, a host-to-device and a
+    device-to-host copy in flight at the same time on two streams: the ceiling of the end-to-end leg."""
+    n = min(pinned_src.numel() * pinned_src.element_size(), pinned_dst.numel() * pinned_dst.element_size())
+    src = pinned_src.view(torch.uint8)[:n]
+    dst = pinned_dst.view(torch.uint8)[:n]
+    d_in = torch.empty(n, dtype=torch.uint8, device="cuda")
+    d_out = torch.empty(n, dtype=torch.uint8, device="cuda")
+    up, down = torch.cuda.Stream(), torch.cuda.Stream()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    torch.cuda.synchronize()
+    for timed in (False, True):
+        if timed:
+            ev[0].record(up)
+            ev[2].record(down)
+        for _ in range(reps if timed else 1):
+            with torch.cuda.stream(up):
+                d_in.copy_(src, non_blocking=True)
+            with torch.cuda.stream(down):
+                dst.copy_(d_out, non_blocking=True)
+        if timed:
+            ev[1].record(up)
+            ev[3].record(down)
+        torch.cuda.synchronize()
+    return {"h2d_gbs": n * reps / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9,
+            "d2h_gbs": n * reps / (ev[2].elapsed_time(ev[3]) * 1e-3) / 1e9,
+            "how": "plain copies of one %.0f MB pinned buffer each way at the same time, %d repetitions" % (n / 1e6, reps)}
+
+
 def cpu_model():
     try:
         with open("/proc/cpuinfo") as f:
@@ -638,7 +667,7 @@ def run_ours(args, w):
                           "shape, no arithmetic; its tables hold 64 of each"}
         del extra, srcs, dsts
 
-    e2e_ms, e2e_steps, h0, h1 = float('nan'), 0, None, None
+    e2e_ms, e2e_steps, h0, h1, link = float('nan'), 0, None, None, None
     no_e2e = args.kernel_only or bool(args.tree)   # a leaf's relay has no host-buffer form: the tree is measured on the device
     if not no_e2e:
         # end to end through the C interface with host buffers: gradients travel host -> device inside
@@ -689,6 +718,8 @@ def run_ours(args, w):
         h1 = ps2.counters()
         e2e_ms = s2.elapsed_time(e2)
         ps2.close()
+        # what the host link gives plain copies of the same buffers, both directions at once
+        link = link_probe(torch, hg[0], hdst[0]) if N > (1 << 24) else None
         del hg, hdst
 
     ms, e2e_ms = replicas.max_over_ranks([ms, e2e_ms], device="cuda")
@@ -843,6 +874,9 @@ def run_ours(args, w):
                 "value": replicas.whole_job_rate(e2e_steps, world, e2e_ms), "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": (h1["h2d_bytes"] - h0["h2d_bytes"]) // e2e_steps,
                 "d2h_bytes_per_step": (h1["d2h_bytes"] - h0["d2h_bytes"]) // e2e_steps,
+                "link": None if not link else dict(
+                    link, achieved_h2d_gbs=(h1["h2d_bytes"] - h0["h2d_bytes"]) / (e2e_ms * 1e-3) / 1e9,
+                    achieved_d2h_gbs=(h1["d2h_bytes"] - h0["d2h_bytes"]) / (e2e_ms * 1e-3) / 1e9),
             },
             "roofline": {
                 "kernel": label,
