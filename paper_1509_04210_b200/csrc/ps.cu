@@ -106,6 +106,7 @@ struct rudra_ps {
   std::vector<void*> slots;        // staging buffers for gradients pushed from host memory
   std::vector<cudaEvent_t> slot_ready;   // upload into the slot has finished
   std::vector<cudaEvent_t> slot_spent;   // the update that read the slot has finished
+  std::vector<uint8_t> slot_upload_unread;   // an upload filled the slot and no launch has waited for it yet
   std::vector<int> free_slots;
   struct DownBuf { float* buf = nullptr; cudaEvent_t filled = nullptr, drained = nullptr; };
   std::vector<DownBuf> down;       // snapshots on their way to host memory
@@ -176,6 +177,7 @@ int free_staging(rudra_ps* ps) {
   ps->slots.clear();
   ps->slot_ready.clear();
   ps->slot_spent.clear();
+  ps->slot_upload_unread.clear();
   ps->free_slots.clear();
   return 0;
 }
@@ -221,6 +223,7 @@ cudaError_t acquire_slot(rudra_ps* ps, int* slot, bool* fresh) {
   ps->slots.push_back(buf);
   ps->slot_ready.push_back(ready);
   ps->slot_spent.push_back(spent);
+  ps->slot_upload_unread.push_back(0);
   *slot = (int)ps->slots.size() - 1;
   *fresh = true;
   return cudaSuccess;
@@ -229,11 +232,21 @@ cudaError_t acquire_slot(rudra_ps* ps, int* slot, bool* fresh) {
 // COPY push mode (Section 3.2: the push message carries the gradient itself): the vector is copied
 // into a staging slot on the handle's stream at push time, so the caller's buffer is free again
 // for anything ordered after this call on that stream.  The slot's last reader ran on the same
-// stream, so the copy needs no event.
+// stream, so the copy needs no event -- unless the slot was filled by an upload that was dropped
+// unread (rudra_ps_set_weights / import_state with gradients still queued): that upload may still
+// be in flight on the upload stream.
 int stage_device_copy(rudra_ps* ps, const void* src, int* slot) {
   bool fresh = false;
   cudaError_t e = acquire_slot(ps, slot, &fresh);
   if (e != cudaSuccess) return cuda_fail(e, "staging buffer allocation");
+  if (ps->slot_upload_unread[*slot]) {
+    e = cudaStreamWaitEvent(ps->stream, ps->slot_ready[*slot], 0);
+    if (e != cudaSuccess) {
+      ps->free_slots.push_back(*slot);
+      return cuda_fail(e, "cudaStreamWaitEvent");
+    }
+    ps->slot_upload_unread[*slot] = 0;
+  }
   e = cudaMemcpyAsync(ps->slots[*slot], src, ps->grad_bytes(), cudaMemcpyDeviceToDevice, ps->stream);
   if (e != cudaSuccess) {
     ps->free_slots.push_back(*slot);
@@ -331,6 +344,7 @@ void append_update(rudra_ps* ps, Window& w) {
       if (e.uploaded) {   // the kernel starts after its uploads
         const cudaError_t we = cudaStreamWaitEvent(ps->stream, ps->slot_ready[e.slot], 0);
         if (we != cudaSuccess && w.wait_error == cudaSuccess) w.wait_error = we;
+        ps->slot_upload_unread[e.slot] = 0;
       }
       w.used_slots.push_back(e.slot);
     }
@@ -681,6 +695,7 @@ int64_t rudra_ps_push_host(rudra_ps* ps, const void* grad_host, uint64_t pulled_
       return cuda_fail(e, "gradient host-to-device copy");
     }
     ps->counters[4] += ps->grad_bytes();
+    ps->slot_upload_unread[slot] = 1;
     return enqueue(ps, ps->slots[slot], pulled_ts, slot, true);
   });
 }

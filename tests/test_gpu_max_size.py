@@ -28,6 +28,7 @@ def test_update_pull_and_leaf_average_beyond_four_giga_weights():
     import torch
     from paper_1509_04210_b200 import binding as rb
 
+    torch.cuda.empty_cache()                                   # blocks cached by earlier tests count as free
     free, _ = torch.cuda.mem_get_info()
     need = N_HUGE * (4 + 4 + 4 + 4 + 4 + 2 * 3) + (2 << 30)   # weights, state, a temporary, slot, average, 3 bf16 gradients
     if free < need:
@@ -98,3 +99,5 @@ def test_update_pull_and_leaf_average_beyond_four_giga_weights():
     assert rel_err(to_host(slot[idx_d]), o2.pull()[0]) <= REL_ONE_STEP
     np.testing.assert_array_equal(root.last_messages()["step"].view(np.uint32), o2.last_messages()["step"].view(np.uint32))
     root.close()
+    del avg, slot, grads
+    torch.cuda.empty_cache()                                   # give the 100 GB back before the next test

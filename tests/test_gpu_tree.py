@@ -301,6 +301,38 @@ def test_group_messages_that_do_not_fit_are_refused():
     gpu.close()
 
 
+def test_copy_push_into_a_slot_whose_upload_was_dropped_unread():
+    """Gradients pushed from host memory are still on their way when set_weights drops the queue; the
+    COPY-mode pushes that follow reuse those staging slots and must not be overtaken by the uploads."""
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    N, lam, n = 1000003, 6, 2
+    rb, gpu, cpus = _pair(N, lam, n, ora.LR_PAPER_N, ora.OPT_MOMENTUM_SGD, 0.9, 5e-4)
+    cpu = cpus[0]
+    junk = [torch.full((N,), 1e30).pin_memory() for _ in range(3)]
+    th0 = synth.initial_weights(N, 0.01, 9)
+    for rounds in range(3):
+        for j in junk:                                        # uploads nobody will read
+            gpu.push_host(j, 0)
+        gpu.set_weights(to_device(th0))                       # drops them; timestamps start over
+        cpu.set_weights(th0)
+        gpu.set_option(rb.OPT_PUSH_MODE, rb.PUSH_COPY)
+        gs = [_grad(N, l, rounds, synth.GRAD_F32) for l in range(3)]
+        scratch = torch.empty(N, device="cuda")
+        for g in gs:
+            scratch.copy_(to_device(g))
+            gpu.push(scratch, 0)
+            cpu.push(g, 0)
+            scratch.fill_(float("nan"))
+        assert gpu.step() == 1 and cpu.step() == 1
+        th, _ = _state(gpu, N)
+        assert np.isfinite(th).all()
+        assert rel_err(th, cpu.pull()[0]) <= REL_ONE_STEP
+        gpu.set_option(rb.OPT_PUSH_MODE, rb.PUSH_BORROW)
+    gpu.close()
+
+
 @pytest.mark.parametrize("N", [70003, 300011])
 def test_copy_push_mode_lets_the_caller_overwrite_its_buffer(N):
     """Section 3.2's push message carries the gradient: with RUDRA_PUSH_COPY the server owns a copy
