@@ -542,6 +542,7 @@ def launch_shapes(w, N, W, region):
 
 
 def run_ours(args, w):
+    global ADAGRAD
     import torch
     import torch.distributed as dist
     from paper_1509_04210_b200 import binding as rb
@@ -731,10 +732,19 @@ def run_ours(args, w):
         del bufs, slots
         torch.cuda.empty_cache()
         others = {}
-        for name, osteps, owarm in (("cifar10", 6000, 300), ("stress", 40, 4), ("imagenet72m", 180, 18)):
-            ow = synth.WORKLOADS[name]
-            orun = DeviceRun(rb, torch, ow, args, seed, stream)
-            oW = default_window(ow)
+        for name, osteps, owarm in (("cifar10", 6000, 300), ("stress", 40, 4), ("imagenet72m", 180, 18),
+                                    ("imagenet_zero_copy_pulls", 360, 18), ("imagenet_adagrad", 360, 18)):
+            # the last two: the default workload with learners sharing weight versions by pointer
+            # (rudra_ps_enable_views) and with AdaGrad at the server (Section 5.5)
+            oviews = name == "imagenet_zero_copy_pulls"
+            was_adagrad, ADAGRAD = ADAGRAD, ADAGRAD or name == "imagenet_adagrad"
+            ow = w if name.startswith("imagenet_") else synth.WORKLOADS[name]
+            if name == "imagenet_adagrad":
+                import dataclasses
+
+                ow = dataclasses.replace(ow, momentum=0.0)
+            orun = DeviceRun(rb, torch, ow, args, seed, stream, views=oviews)
+            oW = default_window(ow, oviews)
             owin = make_windows(ow, -(-owarm // oW) * oW + osteps)
             reg = timed_region(orun, ow, owin, owarm, osteps, oW, barrier)
             og = 2 if ow.grad_dtype == synth.GRAD_BF16 else 4
@@ -753,6 +763,7 @@ def run_ours(args, w):
             del og, osb
             orun.close()
             del orun
+            ADAGRAD = was_adagrad
             torch.cuda.empty_cache()
         # the same ImageNet-scale stream behind the two-level server tree of Section 3.3 (18 leaves of 3
         # learners on this GPU, their averaging fused into the root's launch), and the leaf's own kernel

@@ -88,7 +88,10 @@ rudra_ps* rudra_ps_create(uint64_t nparams, uint32_t lambda, uint32_t n,
 void rudra_ps_destroy(rudra_ps* ps);
 
 /* All later device work of this handle goes to cuda_stream (a cudaStream_t / CUstream value,
- * e.g. torch.cuda.Stream().cuda_stream); NULL selects the legacy default stream. */
+ * e.g. torch.cuda.Stream().cuda_stream); NULL selects the legacy default stream.  The call does
+ * not wait for or order anything: work already enqueued on the previous stream (updates, copies
+ * of queued COPY-mode gradients) must have finished, or the caller must make the new stream wait
+ * for it, before the next call that touches the device. */
 int rudra_ps_set_stream(rudra_ps* ps, void* cuda_stream);
 
 /* Sets one RUDRA_OPT_* key.  Only legal while no gradient is queued (else RUDRA_E_STATE).
