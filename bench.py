@@ -732,7 +732,8 @@ def run_ours(args, w):
         del bufs, slots
         torch.cuda.empty_cache()
         others = {}
-        for name, osteps, owarm in (("cifar10", 6000, 300), ("stress", 40, 4), ("imagenet72m", 180, 18),
+        for name, osteps, owarm in (("tiny", 2000, 100), ("cifar10", 6000, 300), ("mid", 800, 40), ("stress", 40, 4),
+                                    ("imagenet72m", 180, 18),
                                     ("imagenet_zero_copy_pulls", 360, 18), ("imagenet_adagrad", 360, 18)):
             # the last two: the default workload with learners sharing weight versions by pointer
             # (rudra_ps_enable_views) and with AdaGrad at the server (Section 5.5)
