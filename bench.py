@@ -575,6 +575,8 @@ def run_ours(args, w):
         raise SystemExit("--tree is served through rudra_ps_run_events: use --window >= 1")
     run = DeviceRun(rb, torch, w, args, seed, stream, views, args.tree)
     ps, bufs, slots, nbufs = run.ps, run.bufs, run.slots, run.nbufs
+    # smallest power of two that every gradient buffer and slot starts on (full speed needs 1 KB)
+    buf_align = min([(t.data_ptr() & -t.data_ptr()) for t in bufs + slots] + [1 << 21])
     warm_done = args.warmup if W == 0 else -(-args.warmup // W) * W
     extra_steps = 0 if (W == 0 or views or args.tree) else min(args.steps, 216)
     # a short timed region holds few full-window launches: after it, finish the learners' round and
@@ -858,6 +860,7 @@ def run_ours(args, w):
         cfg = workload_config(w)
         cfg["parallelism"] = "replicas x%d (one independent server per GPU)" % world
         cfg["window"] = W
+        cfg["buffer_alignment_bytes"] = buf_align
         cfg["warmup_done"] = region["warmup_done"]
         cfg["launches_timed_every"] = region["launches_sampled_every"]
         cfg["pull"] = ("zero-copy: learners share a pointer to the version they pulled (rudra_ps_enable_views)" if views
