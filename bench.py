@@ -207,9 +207,10 @@ def visible_gpu_index(local_rank):
 # ---------------------------------------------------------------------------------------------
 # CPU oracle legs (the reported baseline and the --impl reference arm)
 # ---------------------------------------------------------------------------------------------
-def oracle_run(w, windows, nsample, grads_host, warmup=0, budget_s=None, max_windows=None, adagrad=False):
+def oracle_run(w, windows, nsample, grads_host, warmup=0, budget_s=None, max_windows=None, adagrad=False, keep=None):
     """Times the oracle, as it stands, over event windows (from the start of the event stream) on
-    the first nsample weights; the first ``warmup`` windows run untimed."""
+    the first nsample weights; the first ``warmup`` windows run untimed.  keep: a list that receives
+    the oracle server, so that the caller can compare its weights with the library's."""
     from oracle import rudra_oracle as ora
 
     ps = ora.OraclePS(nsample, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
@@ -236,7 +237,10 @@ def oracle_run(w, windows, nsample, grads_host, warmup=0, budget_s=None, max_win
             break
         if budget_s is not None and time.perf_counter() - t0 >= budget_s:
             break
-    return done, time.perf_counter() - t0
+    dt = time.perf_counter() - t0
+    if keep is not None:
+        keep.append(ps)
+    return done, dt
 
 
 def oracle_run_all_cores(w, windows, grads_host, cores, budget_s, adagrad=False):
@@ -350,6 +354,47 @@ def link_probe(torch, pinned_src, pinned_dst, reps=6):
     return {"h2d_gbs": n * reps / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9,
             "d2h_gbs": n * reps / (ev[2].elapsed_time(ev[3]) * 1e-3) / 1e9,
             "how": "plain copies of one %.0f MB pinned buffer each way at the same time, %d repetitions" % (n / 1e6, reps)}
+
+
+def parity_with_oracle(rb, torch, w, windows, grads_host, oracle_ps, W, stream):
+    """Runs ``windows`` (from the start of the event stream) through the library on device copies of
+    the oracle's own inputs and compares the whole weight and state vectors with the oracle's."""
+    N = w.nparams
+    ps = rb.ParameterServer(N, w.lam, w.n, w.alpha0, w.momentum, w.weight_decay)
+    ps.set_option(rb.OPT_GRAD_DTYPE, w.grad_dtype)
+    if ADAGRAD:
+        ps.set_option(rb.OPT_OPTIMIZER, rb.OPTIM_ADAGRAD)
+    ps.set_weights(torch.from_numpy(synth.initial_weights(N, w.theta_std)).cuda())
+    ps.sync()
+    ps.set_stream(stream)
+    dev = [torch.from_numpy(g.view(np.int16) if g.dtype == np.uint16 else g).cuda() for g in grads_host]
+    slots = [torch.empty(N, dtype=torch.float32, device="cuda") for _ in range(len(dev))]
+    gtable = rb.pointer_table([dev[l % len(dev)] for l in range(w.lam)])
+    stable = rb.pointer_table([slots[l % len(slots)] for l in range(w.lam)])
+    step = max(W, 1)
+    updates = 0
+    for i in range(0, len(windows), step):
+        chunk = np.concatenate(windows[i:i + step])
+        updates += ps.run_events(chunk, gtable, stable, W)
+    th = torch.empty(N, dtype=torch.float32, device="cuda")
+    st = torch.empty(N, dtype=torch.float32, device="cuda")
+    ps.export_state(th, st)
+    ps.sync()
+
+    def rel(got, want):
+        want = want.astype(np.float64)
+        den = np.maximum(np.abs(want), max(float(np.sqrt(np.mean(want * want))), 1e-30))
+        return float(np.max(np.abs(got.astype(np.float64) - want) / den))
+
+    want_th, ts = oracle_ps.pull()
+    out = {"updates": updates, "weights_compared": N, "max_rel_err_weights": rel(th.cpu().numpy(), want_th),
+           "max_rel_err_state": rel(st.cpu().numpy(), oracle_ps.state()) if (w.momentum != 0.0 or ADAGRAD) else None,
+           "timestamps_equal": int(ts) == ps.timestamp() == updates,
+           "bar": 1e-5 if updates == 1 else 1e-4,
+           "error": "|library - oracle| / max(|oracle|, rms(oracle)), maximum over the vector",
+           "how": "the windows the timed oracle just handled, through rudra_ps_run_events on device copies of the same inputs"}
+    ps.close()
+    return out
 
 
 def cpu_model():
@@ -930,14 +975,20 @@ def run_ours(args, w):
             grads = [t.cpu().numpy() if w.grad_dtype == synth.GRAD_F32 else t.view(torch.int16).cpu().numpy().view(np.uint16)
                      for t in hostg]
             del hostg
+            kept = []
             done, dt = oracle_run(w, windows, N, grads, warmup=1, budget_s=12.0, max_windows=args.steps,
-                                  adagrad=args.optimizer == "adagrad")
+                                  adagrad=args.optimizer == "adagrad", keep=kept)
             line["cpu_baseline"] = {
                 "value": done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
                 "sample": "%d full-size update windows of the same event stream (%d distinct gradient buffers), %.1f s"
                           % (done, nh, dt),
                 "host_cores_available": os.cpu_count(), "cpu_model": cpu_model(),
             }
+            # The windows the oracle just went through, once more through the library on the same
+            # bytes: every weight and every state value of the full-size vector compared.
+            if not args.tree:   # (the tree's events have no flat-server replay in the timed oracle loop)
+                line["cpu_baseline"]["parity"] = parity_with_oracle(rb, torch, w, windows[: done + 1], grads, kept[0], W, stream)
+            del kept
             cores = os.cpu_count() or 1
             if cores > 1:
                 done_all, dt_all = oracle_run_all_cores(w, windows, grads, cores, 8.0, adagrad=args.optimizer == "adagrad")
