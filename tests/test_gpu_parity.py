@@ -446,3 +446,74 @@ def test_one_very_late_gradient_does_not_grow_the_histogram():
     assert len(hist) == rb.HIST_BINS and hist[-1] == 1 and hist[0] == 1 and hist.sum() == 2
     assert ps.last_clock()["sigma"][0] == 0
     ps.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+def test_mixed_message_kinds_in_one_stream(seed):
+    """Every way a gradient can arrive, mixed at random inside the same groups: borrowed device
+    buffers, device buffers copied at push time, host buffers uploaded on the side stream; pulls to
+    device slots and to host memory in between.  Weights and state must equal the oracle's fp32
+    evaluation bit for bit after every update, and be within the bar of its double evaluation."""
+    import torch
+    from paper_1509_04210_b200 import binding as rb
+
+    rng = np.random.default_rng(1000 + seed)
+    N = int(rng.choice([70001, 262144 + 9, 1000003]))
+    lam, n = [(6, 2), (8, 2), (12, 4), (5, 1)][seed - 1]
+    c = lam // n
+    th0 = synth.initial_weights(N, 0.01, seed)
+    gpu = rb.ParameterServer(N, lam, n, 0.03, 0.9, 5e-4)
+    gpu.set_option(rb.OPT_LR_POLICY, rb.LR_PER_GRADIENT)
+    gpu.set_weights(to_device(th0))
+    cpus = []
+    for strict in (False, True):
+        o = ora.OraclePS(N, lam, n, 0.03, 0.9, 5e-4)
+        o.set_policy(ora.LR_PER_GRADIENT)
+        o.set_strict(strict)
+        o.set_weights(th0)
+        cpus.append(o)
+    th = torch.empty(N, device="cuda")
+    st = torch.empty(N, device="cuda")
+    slot = torch.empty(N, device="cuda")
+    host_dst = torch.empty(N).pin_memory()
+    scratch = torch.empty(N, device="cuda")
+    keep = []
+    for upd in range(1, 9):
+        copy_mode = bool(rng.integers(0, 2))                  # the push mode may only change between groups
+        gpu.set_option(rb.OPT_PUSH_MODE, rb.PUSH_COPY if copy_mode else rb.PUSH_BORROW)
+        for l in range(c):
+            g = synth.gradient(N, l, upd, 1e-2, seed=seed)
+            p = int(rng.integers(max(0, upd - 3), upd))        # staleness 0, 1 or 2
+            if rng.integers(0, 2):
+                pinned = torch.from_numpy(g).pin_memory()
+                keep.append(pinned)
+                gpu.push_host(pinned, p)
+            elif copy_mode:
+                scratch.copy_(to_device(g))
+                gpu.push(scratch, p)
+                scratch.fill_(float("nan"))
+            else:
+                d = to_device(g)
+                keep.append(d)
+                gpu.push(d, p)
+            for o in cpus:
+                o.push(g, p)
+            if rng.integers(0, 3) == 0:                        # a pull while the group is open
+                assert gpu.pull(slot) == upd - 1
+        if rng.integers(0, 2):
+            assert gpu.step_pull_many([slot]) == 1
+        else:
+            assert gpu.step() == 1
+            if rng.integers(0, 2):
+                assert gpu.pull_host(host_dst) == upd
+        for o in cpus:
+            assert o.step() == 1
+        gpu.export_state(th, st)
+        gpu.sync()
+        g_clock, o_clock = gpu.last_clock(), cpus[0].last_clock()
+        np.testing.assert_array_equal(g_clock["sigma"], o_clock["sigma"])
+        np.testing.assert_array_equal(g_clock["scale"].view(np.uint32), o_clock["scale"].view(np.uint32))
+        np.testing.assert_array_equal(to_host(th), cpus[1].pull()[0])
+        np.testing.assert_array_equal(to_host(st), cpus[1].state())
+        assert rel_err(to_host(th), cpus[0].pull()[0]) <= (REL_ONE_STEP if upd == 1 else REL_100_STEPS)
+    gpu.close()
