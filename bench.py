@@ -506,6 +506,12 @@ class DeviceRun:
         self.bufs, self.slots = [], []
 
 
+def rounded_warmup(warmup, W):
+    """Warm-up windows really run: whole backlogs, so that the timed backlogs start where a round of
+    the learners starts, and at least two of them (the first launches after set-up run 1-2 % slow)."""
+    return warmup if W == 0 else max(2, -(-warmup // W)) * W
+
+
 def timed_region(run, w, windows, warmup, steps, W, barrier, sampler_factory=None):
     """Warm-up, then exactly ``steps`` update windows between two events.  With a backlog size W the
     warm-up is rounded up to whole backlogs so that the timed backlogs start where a round of the
@@ -514,7 +520,7 @@ def timed_region(run, w, windows, warmup, steps, W, barrier, sampler_factory=Non
     formed from those); for L2-resident, launch-bound workloads only every eighth call is, so that
     the event records do not slow the host loop that is the bottleneck there."""
     torch, stream, ps = run.torch, run.stream, run.ps
-    warm = warmup if W == 0 else -(-warmup // W) * W
+    warm = rounded_warmup(warmup, W)
     wins = windows[: warm + steps]
     assert len(wins) == warm + steps
     if W == 0:
@@ -622,7 +628,7 @@ def run_ours(args, w):
     ps, bufs, slots, nbufs = run.ps, run.bufs, run.slots, run.nbufs
     # smallest power of two that every gradient buffer and slot starts on (full speed needs 1 KB)
     buf_align = min([(t.data_ptr() & -t.data_ptr()) for t in bufs + slots] + [1 << 21])
-    warm_done = args.warmup if W == 0 else -(-args.warmup // W) * W
+    warm_done = rounded_warmup(args.warmup, W)
     extra_steps = 0 if (W == 0 or views or args.tree) else min(args.steps, 216)
     # a short timed region holds few full-window launches: after it, finish the learners' round and
     # time ten more full backlogs, reported beside the roofline (not part of `value`)
@@ -793,7 +799,7 @@ def run_ours(args, w):
                 ow = dataclasses.replace(ow, momentum=0.0)
             orun = DeviceRun(rb, torch, ow, args, seed, stream, views=oviews)
             oW = default_window(ow, oviews)
-            owin = make_windows(ow, -(-owarm // oW) * oW + osteps)
+            owin = make_windows(ow, rounded_warmup(owarm, oW) + osteps)
             reg = timed_region(orun, ow, owin, owarm, osteps, oW, barrier)
             og = 2 if ow.grad_dtype == synth.GRAD_BF16 else 4
             osb = 16 if ow.momentum else 8
@@ -818,7 +824,7 @@ def run_ours(args, w):
         k = 3
         trun = DeviceRun(rb, torch, w, args, seed, stream, fanin=k)
         tsteps, twarm = 360, W
-        treg = timed_region(trun, w, make_windows(w, twarm + tsteps, fanin=k), twarm, tsteps, W, barrier)
+        treg = timed_region(trun, w, make_windows(w, rounded_warmup(twarm, W) + tsteps, fanin=k), twarm, tsteps, W, barrier)
         tbytes = path_bytes_of(w, N, treg)
         avg = torch.empty(N, dtype=torch.float32, device="cuda")
         for i in range(3):
